@@ -1,0 +1,24 @@
+import os
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+
+def pytest_configure(config):
+    config.addinivalue_line("markers", "gpu: needs a CUDA device (run on a B200)")
+
+
+@pytest.fixture(scope="session")
+def oracle32():
+    import oracle
+    return oracle.Oracle("f32")
+
+
+@pytest.fixture(scope="session")
+def oracle64():
+    import oracle
+    return oracle.Oracle("f64")

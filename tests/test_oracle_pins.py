@@ -1,0 +1,389 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix.
+
+None of these tests touches the CUDA library.  Each names the passage it
+checks; together a dropped term, a wrong sign, a wrong index or a transposed
+operand anywhere in the oracle fails at least one of them.
+"""
+import math
+import os
+
+import numpy as np
+import pytest
+
+import ef21_inputs as inputs
+import oracle as oracle_mod
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+# ---------------------------------------------------------------------------
+# Objective and gradient (Section 5, Eq. 19)
+# ---------------------------------------------------------------------------
+
+def _read_closed_form_cases():
+    cases = []
+    with open(os.path.join(GOLDEN, "logistic_closed_form.txt")) as fh:
+        for line in fh:
+            if not line.startswith("case"):
+                continue
+            tok = line.split()
+            fields, key = {}, None
+            for t in tok[1:]:
+                if t in ("A", "y", "x", "lam", "f", "grad"):
+                    key = t
+                    fields[key] = []
+                else:
+                    fields[key].append(float(t))
+            cases.append(fields)
+    return cases
+
+
+@pytest.mark.parametrize("case", _read_closed_form_cases())
+def test_loss_and_grad_closed_form(case, oracle64):
+    A = np.array([case["A"]], dtype=np.float32)
+    y = np.array(case["y"], dtype=np.float32)
+    x = np.array(case["x"], dtype=np.float64)
+    lam = case["lam"][0]
+    assert oracle64.local_loss(A, y, x, lam) == pytest.approx(case["f"][0], rel=1e-14, abs=1e-15)
+    np.testing.assert_allclose(oracle64.local_grad(A, y, x, lam), case["grad"], rtol=1e-14, atol=1e-15)
+
+
+def test_grad_matches_central_differences(oracle64):
+    w = inputs.config(0)
+    rng = np.random.default_rng(123)
+    x = rng.standard_normal(w.d) * 0.7
+    for i in range(w.n):
+        Ai = w.A[w.row_offsets[i]:w.row_offsets[i + 1]]
+        yi = w.y[w.row_offsets[i]:w.row_offsets[i + 1]]
+        g = oracle64.local_grad(Ai, yi, x, w.lam)
+        h = 1e-6
+        fd = np.empty(w.d)
+        for j in range(w.d):
+            e = np.zeros(w.d); e[j] = h
+            fd[j] = (oracle64.local_loss(Ai, yi, x + e, w.lam) - oracle64.local_loss(Ai, yi, x - e, w.lam)) / (2 * h)
+        assert np.max(np.abs(fd - g)) <= 1e-8 * max(1.0, np.max(np.abs(g)))
+
+
+def test_loss_and_grad_at_zero(oracle64):
+    # f(0) = log 2 for every shard; grad f_i(0) = -(1/(2 m_i)) A_i^T y_i (regulariser vanishes).
+    w = inputs.config(1)
+    x = np.zeros(w.d)
+    assert oracle64.loss(w.A, w.y, w.row_offsets, x, w.lam) == pytest.approx(math.log(2.0), rel=1e-14)
+    grads = oracle64.all_grads(w.A, w.y, w.row_offsets, x, w.lam)
+    for i in (0, 7, w.n - 1):
+        r0, r1 = w.row_offsets[i], w.row_offsets[i + 1]
+        expect = -(w.A[r0:r1].astype(np.float64).T @ w.y[r0:r1].astype(np.float64)) / (2.0 * (r1 - r0))
+        np.testing.assert_allclose(grads[i], expect, rtol=1e-13, atol=1e-15)
+
+
+def test_loss_is_mean_of_local_losses_with_own_row_counts(oracle64):
+    # Eq. 1: f = (1/n) sum f_i, f_i averaged over its own m_i; uneven shards expose a wrong normaliser.
+    w = inputs.config(0)
+    off = np.array([0, 10, 60, 61, 200], dtype=np.int64)
+    x = np.linspace(-1, 1, w.d)
+    parts = [oracle64.local_loss(w.A[off[i]:off[i + 1]], w.y[off[i]:off[i + 1]], x, w.lam) for i in range(4)]
+    assert oracle64.loss(w.A, w.y, off, x, w.lam) == pytest.approx(np.mean(parts), rel=1e-14)
+    z = w.A[10:60].astype(np.float64) @ x
+    direct = np.mean(np.logaddexp(0.0, -w.y[10:60] * z)) + w.lam * np.sum(x * x / (1 + x * x))
+    assert parts[1] == pytest.approx(direct, rel=1e-13)
+
+
+def test_large_margins_do_not_overflow(oracle64):
+    A = np.array([[1000.0], [1000.0]], dtype=np.float32)
+    y = np.array([1.0, -1.0], dtype=np.float32)
+    x = np.array([1.0])
+    f = oracle64.local_loss(A, y, x, 0.0)
+    g = oracle64.local_grad(A, y, x, 0.0)
+    assert f == pytest.approx(500.0, rel=1e-12)       # (0 + 1000)/2
+    assert g[0] == pytest.approx(500.0, rel=1e-12)    # (0 + 1000)/2
+
+
+# ---------------------------------------------------------------------------
+# Top-k (Section 2.1, Eq. 3)
+# ---------------------------------------------------------------------------
+
+def _brute_topk(v, k):
+    mag = np.abs(v.astype(np.float64))
+    order = np.lexsort((np.arange(v.size), -mag))      # |v| descending, index ascending
+    keep = np.sort(order[:k])
+    return keep.astype(np.int32), v[keep]
+
+
+@pytest.mark.parametrize("d,k", [(1, 1), (7, 3), (64, 4), (1000, 1), (1000, 999), (4096, 517)])
+def test_topk_matches_brute_force(d, k, oracle32):
+    rng = np.random.default_rng(d * 31 + k)
+    v = rng.standard_normal(d).astype(np.float32)
+    v[rng.integers(0, d, size=max(1, d // 5))] = np.float32(0.5)   # plant exact ties
+    idx, val = oracle32.topk(v, k)
+    bi, bv = _brute_topk(v, k)
+    np.testing.assert_array_equal(idx, bi)
+    np.testing.assert_array_equal(val, bv)
+
+
+def test_topk_matches_brute_force_4m(oracle32):
+    v = inputs.stress_vector(4, 0, 1 << 22)
+    k = (1 << 22) // 1000
+    idx, val = oracle32.topk(v, k)
+    bi, bv = _brute_topk(v, k)
+    np.testing.assert_array_equal(idx, bi)
+    np.testing.assert_array_equal(val, bv)
+
+
+def test_topk_tie_rule_and_signed_zero(oracle32):
+    idx, val = oracle32.topk(np.array([2, -2, 2, 1], dtype=np.float32), 2)
+    np.testing.assert_array_equal(idx, [0, 1]); np.testing.assert_array_equal(val, [2, -2])
+    idx, _ = oracle32.topk(np.full(9, -3.0, dtype=np.float32), 4)
+    np.testing.assert_array_equal(idx, [0, 1, 2, 3])
+    v = np.array([0.0, -0.0, 0.0, 5.0, -0.0], dtype=np.float32)
+    idx, val = oracle32.topk(v, 3)                     # fewer non-zeros than k: zeros by lowest index
+    np.testing.assert_array_equal(idx, [0, 1, 3])
+    assert np.signbit(val[1]) and not np.signbit(val[0]) and val[2] == 5.0
+    v = np.array([1e-45, -3e-45, 0.0, 1e-45], dtype=np.float32)   # subnormals order by magnitude
+    idx, _ = oracle32.topk(v, 2)
+    np.testing.assert_array_equal(idx, [0, 1])
+
+
+def test_topk_identity_when_k_equals_d(oracle32):
+    v = np.random.default_rng(5).standard_normal(257).astype(np.float32)
+    idx, val = oracle32.topk(v, v.size)
+    np.testing.assert_array_equal(idx, np.arange(v.size))
+    np.testing.assert_array_equal(val, v)
+
+
+@pytest.mark.parametrize("d,k", [(64, 4), (300, 1), (1000, 250)])
+def test_topk_contraction_bound(d, k, oracle64):
+    # Eq. 3 with alpha = k/d: ||C(v) - v||^2 <= (1 - k/d) ||v||^2, equality for constant magnitude.
+    rng = np.random.default_rng(d + k)
+    for v in (rng.standard_normal(d), rng.standard_t(3, d), np.where(rng.random(d) < 0.5, -1.5, 1.5)):
+        idx, val = oracle64.topk(v, k)
+        c = np.zeros(d); c[idx] = val
+        lhs, rhs = np.sum((c - v) ** 2), (1 - k / d) * np.sum(v ** 2)
+        assert lhs <= rhs * (1 + 1e-12)
+    idx, val = oracle64.topk(np.where(np.arange(d) % 2 == 0, -1.5, 1.5), k)
+    c = np.zeros(d); c[idx] = val
+    v = np.where(np.arange(d) % 2 == 0, -1.5, 1.5)
+    assert np.sum((c - v) ** 2) == pytest.approx((1 - k / d) * np.sum(v ** 2), rel=1e-12)
+
+
+# ---------------------------------------------------------------------------
+# Algorithm 2 (the loop), Algorithm 1, Section 3.1
+# ---------------------------------------------------------------------------
+
+def _read_hand_example():
+    scal, vec = {}, {}
+    with open(os.path.join(GOLDEN, "alg2_hand_example.txt")) as fh:
+        for line in fh:
+            tok = line.split()
+            if not tok or tok[0].startswith("#"):
+                continue
+            if tok[0] in ("n", "d", "k", "gamma"):
+                scal[tok[0]] = float(tok[1])
+            elif tok[0] in ("V1", "V2"):
+                vec[tok[0]] = [float(t) for t in tok[1:]]
+            else:
+                vec[(tok[0], tok[1])] = [float(t) for t in tok[2:]]
+    return scal, vec
+
+
+@pytest.mark.parametrize("precision", ["f32", "f64"])
+def test_alg2_hand_worked_example(precision):
+    o = oracle_mod.Oracle(precision)
+    scal, vec = _read_hand_example()
+    n, d, k = int(scal["n"]), int(scal["d"]), int(scal["k"])
+    V = np.array([vec["V1"], vec["V2"]])
+    st = oracle_mod.State(o, n, d, k, scal["gamma"])
+    st.init_from_grads(V, mode=0)
+    for t in range(4):
+        tag = f"t{t}"
+        np.testing.assert_array_equal(st.x, vec[(tag, "x")])
+        np.testing.assert_array_equal(st.gi[0], vec[(tag, "g1")])
+        np.testing.assert_array_equal(st.gi[1], vec[(tag, "g2")])
+        np.testing.assert_array_equal(st.g, vec[(tag, "g")])
+        if t > 0:
+            np.testing.assert_array_equal(st.idx[:, 0], vec[(tag, "idx")])
+            np.testing.assert_array_equal(st.val[:, 0], vec[(tag, "val")])
+        st.step_grads(V, 1)
+
+
+def test_k_equals_d_is_gradient_descent(oracle64):
+    # Section 5.2: "GD ... can be thought of as EF21 with k = d".
+    w = inputs.config(0)
+    st = oracle_mod.State(oracle64, w.n, w.d, w.d, w.gamma, w.lam, w.A, w.y, w.row_offsets, w.x0)
+    st.init(0)
+    x = w.x0.astype(np.float64)
+    for _ in range(30):
+        grad = oracle64.all_grads(w.A, w.y, w.row_offsets, x, w.lam).mean(axis=0)
+        np.testing.assert_allclose(st.g, grad, rtol=0, atol=1e-14)
+        x = x - w.gamma * grad
+        st.step(1)
+        np.testing.assert_allclose(st.x, x, rtol=0, atol=1e-13)
+        np.testing.assert_allclose(st.gi, oracle64.all_grads(w.A, w.y, w.row_offsets, st.x, w.lam),
+                                   rtol=0, atol=1e-14)
+
+
+def test_k_equals_d_fp32_state_tracks_gradient(oracle32):
+    # In fp32, g + (a - g) differs from a by a couple of ulps at most; init (Top-d of the gradient) is exact.
+    w = inputs.config(0)
+    st = oracle_mod.State(oracle32, w.n, w.d, w.d, w.gamma, w.lam, w.A, w.y, w.row_offsets, w.x0)
+    st.init(0)
+    np.testing.assert_array_equal(st.gi, oracle32.all_grads(w.A, w.y, w.row_offsets, st.x, w.lam))
+    for _ in range(10):
+        st.step(1)
+        grads = oracle32.all_grads(w.A, w.y, w.row_offsets, st.x, w.lam)
+        assert np.max(np.abs(st.gi - grads)) <= 4 * np.finfo(np.float32).eps * np.max(np.abs(grads))
+
+
+def test_single_node_is_algorithm_1(oracle64):
+    # Algorithm 1: x^{t+1} = x^t - gamma g^t;  g^{t+1} = g^t + C(grad f(x^{t+1}) - g^t);  g^0 = C(grad f(x^0)).
+    w = inputs.config(0)
+    off = np.array([0, w.N], dtype=np.int64)
+    k = 3
+    st = oracle_mod.State(oracle64, 1, w.d, k, w.gamma, w.lam, w.A, w.y, off, w.x0)
+    st.init(0)
+
+    def C(v):
+        keep, vals = _brute_topk(v, k)
+        c = np.zeros_like(v); c[keep] = vals
+        return c
+
+    x = w.x0.astype(np.float64)
+    g = C(oracle64.local_grad(w.A, w.y, x, w.lam))
+    for _ in range(25):
+        np.testing.assert_allclose(st.g, g, rtol=0, atol=1e-15)
+        np.testing.assert_allclose(st.gi[0], g, rtol=0, atol=1e-15)
+        x = x - w.gamma * g
+        g = g + C(oracle64.local_grad(w.A, w.y, x, w.lam) - g)
+        st.step(1)
+        np.testing.assert_allclose(st.x, x, rtol=0, atol=1e-14)
+
+
+@pytest.mark.parametrize("mode", [0, 1, 2])
+def test_master_average_and_one_step_distortion(mode, oracle64):
+    # Algorithm 2, last loop line: g^t = (1/n) sum_i g_i^t at every t.
+    # Proof of Lemma 2, third line: ||g_i^{t+1} - grad f_i(x^{t+1})||^2 <= (1 - k/d) ||grad f_i(x^{t+1}) - g_i^t||^2.
+    w = inputs.config(0)
+    st = oracle_mod.State(oracle64, w.n, w.d, w.k, w.gamma, w.lam, w.A, w.y, w.row_offsets, w.x0)
+    st.init(mode)
+    if mode == 1:
+        assert not st.gi.any() and not st.g.any()
+    if mode == 2:
+        np.testing.assert_allclose(st.gi, st.grads(), atol=1e-16)
+    for _ in range(40):
+        gi_old = st.gi.copy()
+        st.step(1)
+        np.testing.assert_allclose(st.g, st.gi.mean(axis=0), rtol=0, atol=1e-14)
+        grads = st.grads()
+        lhs = np.sum((st.gi - grads) ** 2, axis=1)
+        rhs = (1 - w.k / w.d) * np.sum((grads - gi_old) ** 2, axis=1)
+        assert np.all(lhs <= rhs * (1 + 1e-12) + 1e-30)
+        # the message is exactly the compressed difference, and exactly k coordinates moved
+        for i in range(w.n):
+            bi, bv = _brute_topk(grads[i] - gi_old[i], w.k)
+            np.testing.assert_array_equal(st.idx[i], bi)
+            np.testing.assert_allclose(st.val[i], bv, rtol=0, atol=0)
+            changed = np.flatnonzero(st.gi[i] != gi_old[i])
+            assert set(changed) <= set(bi)
+
+
+def test_theorem_1_lyapunov_descent_and_rate(oracle64):
+    # With gamma at the bound of Theorem 1 (Eq. 13) the proof's Lyapunov function
+    # f(x^t) - f_inf + (gamma/(2 theta)) G^t decreases by at least (gamma/2)||grad f(x^t)||^2 per step,
+    # and the averaged squared gradient norm obeys Eq. 14 with f_inf >= 0.
+    w = inputs.config(0)
+    k = 4
+    gamma = inputs.theory_gamma(w.A, w.row_offsets, w.lam, k)
+    alpha = k / w.d
+    theta = 1 - math.sqrt(1 - alpha)
+    st = oracle_mod.State(oracle64, w.n, w.d, k, gamma, w.lam, w.A, w.y, w.row_offsets, w.x0)
+    st.init(0)
+    T = 60
+    f0 = st.loss()
+    _, G0 = oracle64.diagnostics(w.A, w.y, w.row_offsets, st.x, w.lam, st.gi)
+    f_prev, G_prev = f0, G0
+    sq_norms = []
+    for _ in range(T):
+        nrm2, _ = oracle64.diagnostics(w.A, w.y, w.row_offsets, st.x, w.lam, st.gi)
+        sq_norms.append(nrm2)
+        st.step(1)
+        f_new = st.loss()
+        _, G_new = oracle64.diagnostics(w.A, w.y, w.row_offsets, st.x, w.lam, st.gi)
+        lhs = f_new + gamma / (2 * theta) * G_new
+        rhs = f_prev + gamma / (2 * theta) * G_prev - gamma / 2 * nrm2
+        assert lhs <= rhs + 1e-13
+        f_prev, G_prev = f_new, G_new
+    assert np.mean(sq_norms) <= 2 * (f0 - 0.0) / (gamma * T) + G0 / (theta * T)
+
+
+def test_theory_constants_closed_forms():
+    # Section 3.3 and Example 1: sqrt(beta/theta) = sqrt(1-alpha)/(1-sqrt(1-alpha)) = (1+sqrt(1-alpha))/alpha - 1.
+    for alpha in (1 / 300, 4 / 64, 0.5, 0.999):
+        theta = 1 - math.sqrt(1 - alpha)
+        beta = (1 - alpha) / (1 - math.sqrt(1 - alpha))
+        a = math.sqrt(beta / theta)
+        assert a == pytest.approx(math.sqrt(1 - alpha) / (1 - math.sqrt(1 - alpha)), rel=1e-12)
+        assert a == pytest.approx((1 + math.sqrt(1 - alpha)) / alpha - 1, rel=1e-9)
+        assert a <= 2 / alpha - 1
+
+
+@pytest.mark.parametrize("precision", ["f32", "f64"])
+def test_static_input_markov_compressor_end_state(precision):
+    # Section 3.1 with a constant input v^t = V_i and g_i^0 = 0: after t rounds g_i equals V_i on the
+    # t*k coordinates of largest |V_i| (ties to the lower index) and 0 elsewhere -- exactly, since
+    # V - 0 = V and V - V = 0 -- and the distortion ||g_i - V_i||^2 contracts by (1 - k/d) (Eq. 3).
+    o = oracle_mod.Oracle(precision)
+    n, d, k, T = 3, 500, 7, 20
+    V = np.stack([inputs.stress_vector(11, i, d) for i in range(n)]).astype(o.real)
+    st = oracle_mod.State(o, n, d, k, 0.01)
+    st.init(1)
+    x = np.zeros(d, dtype=np.float64)
+    dist_prev = np.sum(V.astype(np.float64) ** 2, axis=1)
+    for t in range(1, T + 1):
+        x = x - 0.01 * st.g.astype(np.float64)
+        st.step_grads(V, 1)
+        for i in range(n):
+            keep, vals = _brute_topk(V[i], t * k)
+            expect = np.zeros(d, dtype=o.real); expect[keep] = vals
+            np.testing.assert_array_equal(st.gi[i], expect)
+        dist = np.sum((st.gi.astype(np.float64) - V) ** 2, axis=1)
+        assert np.all(dist <= (1 - k / d) * dist_prev * (1 + 1e-12))
+        dist_prev = dist
+        np.testing.assert_allclose(st.g, st.gi.astype(np.float64).mean(axis=0), rtol=0,
+                                   atol=1e-5 if precision == "f32" else 1e-14)
+        np.testing.assert_allclose(st.x, x, rtol=0, atol=2e-6 if precision == "f32" else 1e-14)
+
+
+def _fma_f32(a, b, c):
+    """round_to_nearest_even_fp32(a*b + c) from exact rational arithmetic."""
+    from fractions import Fraction
+    q = Fraction(float(a)) * Fraction(float(b)) + Fraction(float(c))
+    f = np.float32(float(q))
+    cands = {float(f), float(np.nextafter(f, np.float32(np.inf))), float(np.nextafter(f, np.float32(-np.inf)))}
+    best = min(cands, key=lambda t: (abs(Fraction(t) - q), int(np.float32(t).view(np.uint32)) & 1))
+    return np.float32(best)
+
+
+def test_fp32_state_updates_are_single_rounded_operations(oracle32):
+    # The fp32 build must perform g_i + c, s*(1/n), g + p and fma(-gamma, g, x) each as one IEEE operation.
+    rng = np.random.default_rng(9)
+    n, d, k = 5, 40, 3
+    V = rng.standard_normal((n, d)).astype(np.float32)
+    st = oracle_mod.State(oracle32, n, d, k, 0.37)
+    st.init_from_grads(V, mode=0)
+    for _ in range(5):
+        gi, g, x = st.gi.copy(), st.g.copy(), st.x.copy()
+        st.step_grads(V, 1)
+        x_expect = np.array([_fma_f32(-np.float32(0.37), g[j], x[j]) for j in range(d)], dtype=np.float32)
+        np.testing.assert_array_equal(st.x, x_expect)
+        s = np.zeros(d, dtype=np.float32); touched = np.zeros(d, dtype=bool)
+        for i in range(n):
+            v = V[i] - gi[i]
+            keep, vals = _brute_topk(v, k)
+            np.testing.assert_array_equal(st.idx[i], keep)
+            np.testing.assert_array_equal(st.val[i], vals)
+            for j, c in zip(keep, vals):
+                gi[i, j] = np.float32(gi[i, j] + c)
+                s[j] = np.float32(s[j] + c); touched[j] = True
+        inv_n = np.float32(1.0) / np.float32(n)
+        g_expect = np.where(touched, (g + (s * inv_n).astype(np.float32)).astype(np.float32), g)
+        np.testing.assert_array_equal(st.gi, gi)
+        np.testing.assert_array_equal(st.g, g_expect)
