@@ -1,0 +1,164 @@
+/*
+ * libef21 -- the data-parallel hot path of EF21 on one GPU, C ABI.
+ *
+ * EF21 (Richtarik, Sokolov, Fatkhullin, "EF21: A New, Simpler, Theoretically
+ * Better, and Practically Faster Error Feedback") keeps on every worker i a
+ * vector g_i and on the master their average g.  One iteration of its
+ * Algorithm 2 is
+ *
+ *     x^{t+1}   = x^t - gamma g^t                        (master, broadcast)
+ *     c_i^t     = C( grad f_i(x^{t+1}) - g_i^t )         (every worker)
+ *     g_i^{t+1} = g_i^t + c_i^t                          (every worker)
+ *     g^{t+1}   = g^t + (1/n) sum_i c_i^t                (master)
+ *
+ * with C the Top-k compressor of Section 2.1 and, for the built-in objective,
+ * f_i the logistic loss with nonconvex regulariser of Section 5, Eq. 19, on
+ * worker i's rows.  The n workers of the paper are n shards resident on one
+ * device; "send" and "broadcast" are device buffers.
+ *
+ * Conventions
+ *   - Every function returns an ef21_status (0 = success) and never throws or
+ *     aborts.  On failure output arguments are left untouched.
+ *   - Pointers named *_dev are device pointers, *_host are host pointers.
+ *   - The library never allocates or frees device memory: the caller owns
+ *     every device buffer, including the workspace handed to ef21_create /
+ *     ef21_topk, and keeps it alive until ef21_destroy / stream completion.
+ *   - All work is enqueued on the stream given at creation and is
+ *     asynchronous unless stated otherwise; calls on one handle must not
+ *     overlap.  Errors detected on the device (a bounded wait that expired)
+ *     are reported by ef21_poll.
+ *   - Vectors are fp32, indices int32, labels fp32 in {-1,+1}.
+ *   - Top-k keeps the k entries of largest |v_j|, comparing the bit patterns
+ *     of |v_j|; equal magnitudes go to the lower index; exactly k (index,
+ *     value) pairs are produced, indices ascending, values with their sign.
+ *   - State updates are single IEEE fp32 operations in a fixed order, so the
+ *     results are reproducible bit for bit from run to run:
+ *       v = grad - g_i;  g_i[j] += c;  s_j = ((0 + c_{i1,j}) + c_{i2,j}) + ...
+ *       over ascending worker index;  g_j += s_j * (1.0f/n);  x_j = fma(-gamma, g_j, x_j).
+ */
+#ifndef EF21_H
+#define EF21_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ef21_ctx ef21_ctx; /* opaque host-side handle */
+
+typedef enum {
+    EF21_OK = 0,
+    EF21_ERR_INVALID_ARG = 1, /* null pointer, size out of range, non-finite scalar */
+    EF21_ERR_STATE = 2,       /* call order violated (e.g. step before init) */
+    EF21_ERR_WORKSPACE = 3,   /* workspace too small or not 256-byte aligned */
+    EF21_ERR_CUDA = 4,        /* a CUDA runtime call failed */
+    EF21_ERR_TIMEOUT = 5,     /* a bounded device-side wait expired */
+    EF21_ERR_NONFINITE = 6,   /* NaN/Inf met where a finite value is required */
+    EF21_ERR_UNSUPPORTED = 7  /* the requested execution path cannot run this shape */
+} ef21_status;
+
+/* How ef21_init chooses g_i^0 (Algorithm 2, input line; Section 3.3 notes that the
+ * theory holds for any g_i^0). */
+enum {
+    EF21_INIT_COMPRESSED = 0, /* g_i^0 = C(grad f_i(x^0)),  g^0 = (1/n) sum_i g_i^0 */
+    EF21_INIT_ZERO = 1,       /* g_i^0 = 0,                 g^0 = 0 */
+    EF21_INIT_GRADIENT = 2    /* g_i^0 = grad f_i(x^0),     g^0 = (1/n) sum_i g_i^0 */
+};
+
+/* Execution paths of ef21_step; results are bit-identical across paths given
+ * bit-identical local gradients. */
+enum {
+    EF21_PATH_AUTO = 0,       /* pick the fastest path that supports the shape */
+    EF21_PATH_LAUNCHES = 1,   /* one kernel launch per stage, any shape */
+    EF21_PATH_PERSISTENT = 2  /* one cooperative kernel for all steps; shards on chip */
+};
+
+const char* ef21_status_string(ef21_status s);
+
+/* Bytes of device workspace ef21_create needs for n workers, dimension d, k kept
+ * entries and total_rows rows over all shards (0 if only supplied gradients are
+ * used).  Returns 0 for invalid arguments (n < 1, d < 1, k < 1, k > d, d >= 2^31,
+ * total_rows < 0). */
+size_t ef21_workspace_bytes(int32_t n, int64_t d, int32_t k, int64_t total_rows);
+
+/* Creates a handle.  workspace_dev: at least ef21_workspace_bytes(...) bytes, 256-byte
+ * aligned, owned by the caller, used exclusively by this handle.  cuda_stream: a
+ * cudaStream_t (NULL = default stream).  gamma > 0 and lambda >= 0 must be finite.
+ * total_rows is the capacity for ef21_load_shards. */
+ef21_status ef21_create(ef21_ctx** out, int32_t n, int64_t d, int32_t k, float gamma, float lambda,
+                        int64_t total_rows, void* workspace_dev, size_t workspace_bytes,
+                        void* cuda_stream);
+void ef21_destroy(ef21_ctx* ctx); /* frees host memory only; NULL is allowed */
+
+/* Worker i owns rows [row_offsets_host[i], row_offsets_host[i+1]) of A (row-major,
+ * leading dimension d) and of y; row_offsets_host has n+1 non-decreasing entries, the
+ * first 0, the last = total_rows given at creation.  A and y are copied into the
+ * workspace (padded row pitch), so the caller may release them once the stream has
+ * passed this call.  The _host variant takes host pointers and issues the
+ * host-to-device copies itself. (Section 5: data split over n clients.) */
+ef21_status ef21_load_shards(ef21_ctx* ctx, const float* A_dev, const float* y_dev,
+                             const int64_t* row_offsets_host);
+ef21_status ef21_load_shards_host(ef21_ctx* ctx, const float* A_host, const float* y_host,
+                                  const int64_t* row_offsets_host);
+
+/* x^0 (default: the zero vector).  d floats. */
+ef21_status ef21_set_x(ef21_ctx* ctx, const float* x0_dev);
+
+/* Algorithm 2, input line: builds g_i^0 and g^0 from the local gradients at x^0
+ * (mode: EF21_INIT_*).  Modes 0 and 2 need shards; mode 1 does not. */
+ef21_status ef21_init(ef21_ctx* ctx, int32_t mode);
+/* The same with caller-supplied local gradients V_dev[n][d] (leading dimension d). */
+ef21_status ef21_init_grads(ef21_ctx* ctx, const float* V_dev, int32_t mode);
+
+/* `steps` iterations of Algorithm 2's loop (x update, local gradients of Eq. 19,
+ * difference, Top-k, g_i update, aggregation).  After init and t steps in total the
+ * state is (x^t, g^t, g_i^t) in the paper's indexing. */
+ef21_status ef21_step(ef21_ctx* ctx, int32_t steps);
+/* The same loop with grad f_i replaced by the caller's V_dev[n][d], re-used unchanged at
+ * each of the `steps` iterations (the static input sequence of Section 3.1); call with
+ * steps = 1 and fresh V for a changing sequence.  V must stay valid until the stream has
+ * passed this call. */
+ef21_status ef21_step_grads(ef21_ctx* ctx, const float* V_dev, int32_t steps);
+
+/* grad f_i(x) for the current x and all workers, written to grads_out_dev[n][d]
+ * (Eq. 19 differentiated; state is not changed). */
+ef21_status ef21_local_grads(ef21_ctx* ctx, float* grads_out_dev);
+
+/* Standalone Top-k compressor (Section 2.1) on `batch` vectors v_dev[batch][d] (leading
+ * dimension d): idx_out_dev[batch][k] ascending, val_out_dev[batch][k].  The workspace
+ * needs ef21_topk_workspace_bytes(batch, d, k) bytes, 256-byte aligned. */
+size_t ef21_topk_workspace_bytes(int32_t batch, int64_t d, int32_t k);
+ef21_status ef21_topk(const float* v_dev, int32_t batch, int64_t d, int32_t k,
+                      int32_t* idx_out_dev, float* val_out_dev,
+                      void* workspace_dev, size_t workspace_bytes, void* cuda_stream);
+
+/* Copies of the state; any pointer may be NULL.  gi is [n][d]; last_idx/last_val are the
+ * most recent messages c_i, [n][k] each.  set_state also marks the handle initialised
+ * (resume / teacher forcing); x, g or gi left NULL keep their current contents. */
+ef21_status ef21_get_state(ef21_ctx* ctx, float* x_dev, float* g_dev, float* gi_dev,
+                           int32_t* last_idx_dev, float* last_val_dev);
+ef21_status ef21_get_state_host(ef21_ctx* ctx, float* x_host, float* g_host, float* gi_host,
+                                int32_t* last_idx_host, float* last_val_host); /* synchronises */
+ef21_status ef21_set_state(ef21_ctx* ctx, const float* x_dev, const float* g_dev, const float* gi_dev);
+
+/* Diagnostics at the current state (synchronises): f(x) of Eq. 19 / Eq. 1, ||grad f(x)||^2,
+ * and G^t = (1/n) sum_i ||g_i - grad f_i(x)||^2 of Section 3.3.  Any pointer may be NULL. */
+ef21_status ef21_eval(ef21_ctx* ctx, double* f, double* grad_norm2, double* G);
+
+/* Synchronises the stream and returns the device status word: EF21_OK, or the first
+ * error a kernel recorded (EF21_ERR_TIMEOUT, EF21_ERR_NONFINITE), or EF21_ERR_CUDA. */
+ef21_status ef21_poll(ef21_ctx* ctx);
+
+/* Forces an execution path (EF21_PATH_*) for later ef21_step calls. */
+ef21_status ef21_set_path(ef21_ctx* ctx, int32_t path);
+/* The path the last ef21_step / ef21_step_grads actually used (EF21_PATH_*), 0 if none yet. */
+int32_t ef21_last_path(const ef21_ctx* ctx);
+/* Kernel launches enqueued by this handle since creation (copies are not counted). */
+int64_t ef21_launch_count(const ef21_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EF21_H */

@@ -1,0 +1,100 @@
+// State updates of Algorithm 2 after the messages c_i = (idx, val)[k] are known:
+//   g_i <- g_i + c_i                      (worker state, node loop)
+//   g   <- g + (1/n) sum_i c_i            (master, last line of the loop)
+//   x   <- x - gamma g                    (master, first line of the loop)
+// The per-coordinate sum over workers runs in ascending worker index starting from 0, each
+// operation a single rounded fp32 add / multiply, so the result does not depend on scheduling.
+#pragma once
+#include "common.cuh"
+
+namespace ef21 {
+
+constexpr int AGG_TILE = 2048;     // coordinates per block in the aggregation
+constexpr int AGG_BLOCK = 256;
+
+// g_i[idx] += val for all n*k message entries (indices within a worker are distinct).
+__global__ void apply_messages_kernel(const int* __restrict__ idx, const float* __restrict__ val,
+                                      i64 total, int k, i64 ld, float* __restrict__ gi) {
+    const i64 e = blockIdx.x * (i64)blockDim.x + threadIdx.x;
+    if (e >= total) return;
+    const i64 i = e / k;
+    float* p = gi + i * ld + idx[e];
+    *p = __fadd_rn(*p, val[e]);
+}
+
+// off[i][b] = first position in worker i's ascending index list with idx >= b * AGG_TILE,
+// for b = 0 .. ntiles (so tile b owns entries [off[i][b], off[i][b+1])).
+__global__ void agg_offsets_kernel(const int* __restrict__ idx, int n, int k, int ntiles,
+                                   int* __restrict__ off) {
+    const i64 e = blockIdx.x * (i64)blockDim.x + threadIdx.x;
+    const i64 total = (i64)n * (ntiles + 1);
+    if (e >= total) return;
+    const int i = (int)(e / (ntiles + 1));
+    const int b = (int)(e - (i64)i * (ntiles + 1));
+    const i64 bound = (i64)b * AGG_TILE;
+    const int* __restrict__ ix = idx + (i64)i * k;
+    int lo = 0, hi = k;
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if ((i64)ix[mid] < bound) lo = mid + 1; else hi = mid;
+    }
+    off[e] = lo;
+}
+
+// One block per tile of AGG_TILE coordinates.  UPDATE_X: also perform x <- fma(-gamma, g_old, x)
+// on the tile before g changes (Algorithm 2 updates x from g^t, then g^{t+1} from the messages).
+template <bool UPDATE_X>
+__global__ void __launch_bounds__(AGG_BLOCK)
+aggregate_kernel(const int* __restrict__ idx, const float* __restrict__ val, const int* __restrict__ off,
+                 int n, int k, int ntiles, i64 d, float inv_n, float gamma,
+                 float* __restrict__ g, float* __restrict__ x) {
+    __shared__ float s[AGG_TILE];
+    __shared__ unsigned char touched[AGG_TILE];
+    const int b = blockIdx.x;
+    const i64 j0 = (i64)b * AGG_TILE;
+    for (int t = threadIdx.x; t < AGG_TILE; t += AGG_BLOCK) { s[t] = 0.f; touched[t] = 0; }
+    __syncthreads();
+    for (int i = 0; i < n; ++i) {
+        const int lo = off[(i64)i * (ntiles + 1) + b], hi = off[(i64)i * (ntiles + 1) + b + 1];
+        for (int e = lo + threadIdx.x; e < hi; e += AGG_BLOCK) {
+            const int t = (int)((i64)idx[(i64)i * k + e] - j0);
+            s[t] = __fadd_rn(s[t], val[(i64)i * k + e]);
+            touched[t] = 1;
+        }
+        __syncthreads();
+    }
+    for (int t = threadIdx.x; t < AGG_TILE; t += AGG_BLOCK) {
+        const i64 j = j0 + t;
+        if (j >= d) break;
+        if (UPDATE_X) {
+            const float gj = g[j];
+            x[j] = fmaf(-gamma, gj, x[j]);
+            if (touched[t]) g[j] = __fadd_rn(gj, __fmul_rn(s[t], inv_n));
+        } else if (touched[t]) {
+            g[j] = __fadd_rn(g[j], __fmul_rn(s[t], inv_n));
+        }
+    }
+}
+
+// x <- fma(-gamma, g, x), elementwise.
+__global__ void x_update_kernel(const float* __restrict__ g, float* __restrict__ x, i64 d, float gamma) {
+    for (i64 j = blockIdx.x * (i64)blockDim.x + threadIdx.x; j < d; j += (i64)gridDim.x * blockDim.x)
+        x[j] = fmaf(-gamma, g[j], x[j]);
+}
+
+// Dense initial state g_i^0 = V_i, g^0_j = ((0 + V_0j) + V_1j + ...) * (1/n): the k = d message
+// round applied to zero state.
+__global__ void dense_init_kernel(const float* __restrict__ V, i64 pitch_v, int n, i64 d, i64 ld,
+                                  float inv_n, float* __restrict__ gi, float* __restrict__ g) {
+    for (i64 j = blockIdx.x * (i64)blockDim.x + threadIdx.x; j < d; j += (i64)gridDim.x * blockDim.x) {
+        float s = 0.f;
+        for (int i = 0; i < n; ++i) {
+            const float v = V[(i64)i * pitch_v + j];
+            gi[(i64)i * ld + j] = __fadd_rn(0.f, v);
+            s = __fadd_rn(s, v);
+        }
+        g[j] = __fadd_rn(0.f, __fmul_rn(s, inv_n));
+    }
+}
+
+}  // namespace ef21

@@ -1,0 +1,80 @@
+// Shared device helpers of libef21 (sm_100a).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace ef21 {
+
+typedef long long i64;
+
+// Status word layout in the workspace (one 256-byte slot): word 0 = first error code seen.
+__device__ __forceinline__ void record_error(unsigned* status, unsigned code) {
+    atomicCAS(status, 0u, code);
+}
+
+// Magnitude key of Top-k: the bit pattern of |v|.  For finite values the order of keys is the
+// order of magnitudes; +0 and -0 share key 0.
+__device__ __forceinline__ unsigned mag_key(float v) { return __float_as_uint(v) & 0x7fffffffu; }
+
+// v = a - b as one rounded fp32 subtraction (b == nullptr: v = a).
+__device__ __forceinline__ float diff_at(const float* __restrict__ a, const float* __restrict__ b, i64 j) {
+    float av = a[j];
+    return b ? __fsub_rn(av, b[j]) : av;
+}
+
+__device__ __forceinline__ unsigned warp_incl_scan(unsigned v) {
+    const unsigned lane = threadIdx.x & 31u;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        unsigned t = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= (unsigned)o) v += t;
+    }
+    return v;
+}
+
+// Exclusive prefix sum over the threads of a block (blockDim.x a multiple of 32, <= 1024).
+// scratch: 33 unsigned words of shared memory.  Returns the exclusive prefix; total = block sum.
+__device__ __forceinline__ unsigned block_excl_scan(unsigned v, unsigned* scratch, unsigned& total) {
+    const unsigned lane = threadIdx.x & 31u, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    __syncthreads();
+    unsigned inc = warp_incl_scan(v);
+    if (lane == 31u) scratch[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        unsigned w = lane < nwarps ? scratch[lane] : 0u;
+        unsigned wi = warp_incl_scan(w);
+        scratch[lane] = wi - w;
+        if (lane == 31u) scratch[32] = wi;
+    }
+    __syncthreads();
+    total = scratch[32];
+    return inc - v + scratch[warp];
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// -y / (1 + exp(y z)): derivative of log(1 + exp(-y z)) with respect to z, overflow-safe.
+__device__ __forceinline__ float logistic_residual(float y, float z) {
+    float t = y * z;
+    float e = expf(-fabsf(t));                 // in (0, 1]
+    float num = t >= 0.f ? e : 1.f;
+    return __fdiv_rn(-y * num, 1.f + e);
+}
+
+// d/dx of lambda x^2/(1+x^2) = 2 lambda x / (1+x^2)^2.
+__device__ __forceinline__ float regulariser_grad(float lambda, float x) {
+    float q = fmaf(x, x, 1.f);
+    return __fdiv_rn(2.f * lambda * x, q * q);
+}
+
+}  // namespace ef21

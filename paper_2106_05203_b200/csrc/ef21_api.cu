@@ -1,0 +1,489 @@
+// libef21: C-ABI entry points (see include/ef21.h) and the host-side orchestration.
+#include "../../include/ef21.h"
+
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "apply.cuh"
+#include "common.cuh"
+#include "grad.cuh"
+#include "topk.cuh"
+
+using namespace ef21;
+
+namespace {
+
+constexpr size_t ALIGN = 256;
+inline size_t align_up(size_t v) { return (v + ALIGN - 1) / ALIGN * ALIGN; }
+inline i64 ceil_div(i64 a, i64 b) { return (a + b - 1) / b; }
+
+// ---------------------------------------------------------------------------------------------
+// Workspace layouts
+// ---------------------------------------------------------------------------------------------
+
+struct TopkLayout {
+    size_t state, hist, chunks, total;
+    int nchunks;
+};
+
+TopkLayout topk_layout(i64 batch, i64 d) {
+    TopkLayout L;
+    L.nchunks = (int)ceil_div(d, TK_CHUNK);
+    size_t o = 0;
+    L.state = o; o += align_up((size_t)batch * sizeof(TkState));
+    L.hist = o; o += align_up((size_t)batch * TK_BINS * sizeof(unsigned));
+    L.chunks = o; o += align_up((size_t)batch * (size_t)L.nchunks * sizeof(uint2));
+    L.total = o;
+    return L;
+}
+
+int grad_tile_rows(i64 N, i64 ld) {
+    i64 cap = 65536 / (ld * 4);
+    if (cap < 1) cap = 1;
+    if (cap > GRAD_TILE_MAX_ROWS) cap = GRAD_TILE_MAX_ROWS;
+    i64 want = ceil_div(N, 4 * 148);
+    if (want < 8) want = 8;
+    return (int)(want < cap ? want : cap);
+}
+
+struct Layout {
+    i64 ld;            // padded vector pitch (floats), multiple of 4
+    int agg_tiles;     // tiles of AGG_TILE coordinates
+    int tile_rows;     // rows per gradient tile
+    i64 max_tiles;     // capacity of the gradient tile table
+    size_t status, x, g, gi, msg_idx, msg_val, topk, agg_off, eval_out;
+    size_t A, y, row_off, tile_begin, tiles, partial, loss_partial, grad;
+    size_t total;
+    TopkLayout tk;
+};
+
+Layout make_layout(i64 n, i64 d, i64 k, i64 N) {
+    Layout L;
+    L.ld = (d + 3) / 4 * 4;
+    L.agg_tiles = (int)ceil_div(d, AGG_TILE);
+    L.tk = topk_layout(n, d);
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t at = o; o += align_up(bytes); return at; };
+    L.status = take(256);
+    L.x = take((size_t)L.ld * 4);
+    L.g = take((size_t)L.ld * 4);
+    L.gi = take((size_t)n * L.ld * 4);
+    L.msg_idx = take((size_t)n * k * 4);
+    L.msg_val = take((size_t)n * k * 4);
+    L.topk = take(L.tk.total);
+    L.agg_off = take((size_t)n * (L.agg_tiles + 1) * 4);
+    L.eval_out = take(256);
+    L.tile_rows = 0; L.max_tiles = 0;
+    L.A = L.y = L.row_off = L.tile_begin = L.tiles = L.partial = L.loss_partial = L.grad = 0;
+    if (N > 0) {
+        L.tile_rows = grad_tile_rows(N, L.ld);
+        L.max_tiles = N / L.tile_rows + n;
+        L.A = take((size_t)N * L.ld * 4);
+        L.y = take((size_t)N * 4);
+        L.row_off = take((size_t)(n + 1) * 8);
+        L.tile_begin = take((size_t)(n + 1) * 4);
+        L.tiles = take((size_t)L.max_tiles * sizeof(RowTile));
+        L.partial = take((size_t)L.max_tiles * L.ld * 4);
+        L.loss_partial = take((size_t)L.max_tiles * 8);
+        L.grad = take((size_t)n * L.ld * 4);
+    }
+    L.total = o;
+    return L;
+}
+
+bool valid_shape(i64 n, i64 d, i64 k, i64 N) {
+    return n >= 1 && d >= 1 && k >= 1 && k <= d && d < ((i64)1 << 31) && N >= 0 && n <= 65535;
+}
+
+}  // namespace
+
+struct ef21_ctx {
+    int n; i64 d; int k; float gamma, lambda; i64 N;
+    cudaStream_t stream;
+    char* ws;
+    Layout L;
+    bool shards_loaded, inited;
+    int num_tiles;
+    int path, last_path;
+    i64 launches;
+    std::vector<i64> row_off;
+    std::vector<RowTile> tiles;
+    std::vector<int> tile_begin;
+
+    template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
+    float* x() const { return at<float>(L.x); }
+    float* g() const { return at<float>(L.g); }
+    float* gi() const { return at<float>(L.gi); }
+    int* msg_idx() const { return at<int>(L.msg_idx); }
+    float* msg_val() const { return at<float>(L.msg_val); }
+    unsigned* status() const { return at<unsigned>(L.status); }
+};
+
+#define CU(call)                                         \
+    do {                                                 \
+        cudaError_t e__ = (call);                        \
+        if (e__ != cudaSuccess) return EF21_ERR_CUDA;    \
+    } while (0)
+#define EF(call)                                         \
+    do {                                                 \
+        ef21_status s__ = (call);                        \
+        if (s__ != EF21_OK) return s__;                  \
+    } while (0)
+
+namespace {
+
+struct TopkBuffers {
+    TkState* state; unsigned* hist; uint2* chunks; int nchunks;
+};
+
+TopkBuffers topk_buffers(char* base, const TopkLayout& L) {
+    TopkBuffers B;
+    B.state = reinterpret_cast<TkState*>(base + L.state);
+    B.hist = reinterpret_cast<unsigned*>(base + L.hist);
+    B.chunks = reinterpret_cast<uint2*>(base + L.chunks);
+    B.nchunks = L.nchunks;
+    return B;
+}
+
+// Exact Top-k of v = a - b for `batch` vectors (b may be null); general multi-block path.
+ef21_status enqueue_topk_general(cudaStream_t st, const float* a, i64 pitch_a, const float* b, i64 pitch_b,
+                                 int batch, i64 d, int k, int* idx_out, float* val_out,
+                                 const TopkBuffers& B, i64* launches) {
+    tk_reset_kernel<<<batch, 256, 0, st>>>(B.state, B.hist, batch, (unsigned)k);
+    dim3 grid((unsigned)B.nchunks, (unsigned)batch);
+    for (int level = 0; level < 3; ++level) {
+        tk_hist_kernel<<<grid, TK_BLOCK, 0, st>>>(a, pitch_a, b, pitch_b, d, level, B.state, B.hist);
+        tk_find_kernel<<<batch, 1024, 0, st>>>(B.state, B.hist, level);
+    }
+    tk_count_kernel<<<grid, TK_BLOCK, 0, st>>>(a, pitch_a, b, pitch_b, d, B.state, B.chunks, B.nchunks);
+    tk_scan_kernel<<<batch, 1024, 0, st>>>(B.chunks, B.nchunks);
+    tk_write_kernel<<<grid, TK_BLOCK, 0, st>>>(a, pitch_a, b, pitch_b, d, B.state, B.chunks, B.nchunks, k,
+                                               idx_out, val_out);
+    if (launches) *launches += 10;
+    CU(cudaGetLastError());
+    return EF21_OK;
+}
+
+ef21_status enqueue_grads(ef21_ctx* c, bool with_loss) {
+    if (c->num_tiles > 0) {
+        grad_tiles_kernel<<<c->num_tiles, GRAD_BLOCK, 0, c->stream>>>(
+            c->at<float>(c->L.A), c->at<float>(c->L.y), c->x(), c->at<RowTile>(c->L.tiles), (int)c->L.ld,
+            c->at<float>(c->L.partial), with_loss ? c->at<double>(c->L.loss_partial) : nullptr);
+        c->launches += 1;
+    }
+    dim3 grid((unsigned)ceil_div(c->L.ld, 256), (unsigned)c->n);
+    grad_finish_kernel<<<grid, 256, 0, c->stream>>>(c->at<float>(c->L.partial), c->at<int>(c->L.tile_begin),
+                                                    c->at<i64>(c->L.row_off), c->x(), c->lambda, (int)c->d,
+                                                    (int)c->L.ld, c->at<float>(c->L.grad));
+    c->launches += 1;
+    CU(cudaGetLastError());
+    return EF21_OK;
+}
+
+// One message round: c_i = C(a_i - g_i), g_i += c_i, g += (1/n) sum c_i (and, if update_x,
+// x <- x - gamma g_old fused into the aggregation).
+ef21_status enqueue_round(ef21_ctx* c, const float* a, i64 pitch_a, bool update_x) {
+    TopkBuffers B = topk_buffers(c->ws + c->L.topk, c->L.tk);
+    EF(enqueue_topk_general(c->stream, a, pitch_a, c->gi(), c->L.ld, c->n, c->d, c->k, c->msg_idx(),
+                            c->msg_val(), B, &c->launches));
+    const i64 total = (i64)c->n * c->k;
+    apply_messages_kernel<<<(unsigned)ceil_div(total, 256), 256, 0, c->stream>>>(c->msg_idx(), c->msg_val(), total,
+                                                                                c->k, c->L.ld, c->gi());
+    const i64 noff = (i64)c->n * (c->L.agg_tiles + 1);
+    agg_offsets_kernel<<<(unsigned)ceil_div(noff, 256), 256, 0, c->stream>>>(c->msg_idx(), c->n, c->k,
+                                                                            c->L.agg_tiles, c->at<int>(c->L.agg_off));
+    const float inv_n = 1.0f / (float)c->n;
+    if (update_x)
+        aggregate_kernel<true><<<c->L.agg_tiles, AGG_BLOCK, 0, c->stream>>>(
+            c->msg_idx(), c->msg_val(), c->at<int>(c->L.agg_off), c->n, c->k, c->L.agg_tiles, c->d, inv_n,
+            c->gamma, c->g(), c->x());
+    else
+        aggregate_kernel<false><<<c->L.agg_tiles, AGG_BLOCK, 0, c->stream>>>(
+            c->msg_idx(), c->msg_val(), c->at<int>(c->L.agg_off), c->n, c->k, c->L.agg_tiles, c->d, inv_n,
+            c->gamma, c->g(), c->x());
+    c->launches += 3;
+    CU(cudaGetLastError());
+    return EF21_OK;
+}
+
+ef21_status enqueue_x_update(ef21_ctx* c) {
+    const unsigned blocks = (unsigned)std::min<i64>(ceil_div(c->d, 256), 148 * 8);
+    x_update_kernel<<<blocks, 256, 0, c->stream>>>(c->g(), c->x(), c->d, c->gamma);
+    c->launches += 1;
+    CU(cudaGetLastError());
+    return EF21_OK;
+}
+
+ef21_status zero_state(ef21_ctx* c) {
+    CU(cudaMemsetAsync(c->gi(), 0, (size_t)c->n * c->L.ld * 4, c->stream));
+    CU(cudaMemsetAsync(c->g(), 0, (size_t)c->L.ld * 4, c->stream));
+    return EF21_OK;
+}
+
+ef21_status init_from(ef21_ctx* c, const float* V, i64 pitch, int mode) {
+    EF(zero_state(c));
+    if (mode == EF21_INIT_COMPRESSED) {
+        EF(enqueue_round(c, V, pitch, false));
+    } else if (mode == EF21_INIT_GRADIENT) {
+        const unsigned blocks = (unsigned)std::min<i64>(ceil_div(c->d, 256), 148 * 8);
+        dense_init_kernel<<<blocks, 256, 0, c->stream>>>(V, pitch, c->n, c->d, c->L.ld, 1.0f / (float)c->n,
+                                                        c->gi(), c->g());
+        c->launches += 1;
+        CU(cudaGetLastError());
+    }
+    c->inited = true;
+    return EF21_OK;
+}
+
+ef21_status finish_load(ef21_ctx* c, const i64* row_offsets_host) {
+    // Validate and build the tile table.
+    if (row_offsets_host[0] != 0 || row_offsets_host[c->n] != c->N) return EF21_ERR_INVALID_ARG;
+    for (int i = 0; i < c->n; ++i)
+        if (row_offsets_host[i + 1] < row_offsets_host[i]) return EF21_ERR_INVALID_ARG;
+    c->row_off.assign(row_offsets_host, row_offsets_host + c->n + 1);
+    c->tiles.clear();
+    c->tile_begin.assign(c->n + 1, 0);
+    const int R = c->L.tile_rows;
+    for (int i = 0; i < c->n; ++i) {
+        c->tile_begin[i] = (int)c->tiles.size();
+        for (i64 r = c->row_off[i]; r < c->row_off[i + 1]; r += R) {
+            RowTile t;
+            t.row0 = r;
+            t.rows = (int)std::min<i64>(R, c->row_off[i + 1] - r);
+            t.worker = i;
+            c->tiles.push_back(t);
+        }
+    }
+    c->tile_begin[c->n] = (int)c->tiles.size();
+    c->num_tiles = (int)c->tiles.size();
+    if ((i64)c->num_tiles > c->L.max_tiles) return EF21_ERR_WORKSPACE;
+    CU(cudaMemcpyAsync(c->at<i64>(c->L.row_off), c->row_off.data(), (size_t)(c->n + 1) * 8, cudaMemcpyHostToDevice, c->stream));
+    CU(cudaMemcpyAsync(c->at<int>(c->L.tile_begin), c->tile_begin.data(), (size_t)(c->n + 1) * 4, cudaMemcpyHostToDevice, c->stream));
+    if (c->num_tiles > 0)
+        CU(cudaMemcpyAsync(c->at<RowTile>(c->L.tiles), c->tiles.data(), (size_t)c->num_tiles * sizeof(RowTile),
+                           cudaMemcpyHostToDevice, c->stream));
+    c->shards_loaded = true;
+    return EF21_OK;
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------------
+// C ABI
+// ---------------------------------------------------------------------------------------------
+
+extern "C" {
+
+const char* ef21_status_string(ef21_status s) {
+    switch (s) {
+        case EF21_OK: return "ok";
+        case EF21_ERR_INVALID_ARG: return "invalid argument";
+        case EF21_ERR_STATE: return "call order violated";
+        case EF21_ERR_WORKSPACE: return "workspace too small or misaligned";
+        case EF21_ERR_CUDA: return "CUDA runtime error";
+        case EF21_ERR_TIMEOUT: return "bounded device wait expired";
+        case EF21_ERR_NONFINITE: return "non-finite value";
+        case EF21_ERR_UNSUPPORTED: return "shape not supported by the requested path";
+    }
+    return "unknown status";
+}
+
+size_t ef21_workspace_bytes(int32_t n, int64_t d, int32_t k, int64_t total_rows) {
+    if (!valid_shape(n, d, k, total_rows)) return 0;
+    return make_layout(n, d, k, total_rows).total;
+}
+
+ef21_status ef21_create(ef21_ctx** out, int32_t n, int64_t d, int32_t k, float gamma, float lambda,
+                        int64_t total_rows, void* workspace_dev, size_t workspace_bytes, void* cuda_stream) {
+    if (!out || !valid_shape(n, d, k, total_rows)) return EF21_ERR_INVALID_ARG;
+    if (!(gamma > 0.f) || !std::isfinite(gamma) || !(lambda >= 0.f) || !std::isfinite(lambda)) return EF21_ERR_INVALID_ARG;
+    if (!workspace_dev) return EF21_ERR_INVALID_ARG;
+    Layout L = make_layout(n, d, k, total_rows);
+    if (workspace_bytes < L.total || (reinterpret_cast<uintptr_t>(workspace_dev) % ALIGN) != 0) return EF21_ERR_WORKSPACE;
+    ef21_ctx* c = new (std::nothrow) ef21_ctx();
+    if (!c) return EF21_ERR_INVALID_ARG;
+    c->n = n; c->d = d; c->k = k; c->gamma = gamma; c->lambda = lambda; c->N = total_rows;
+    c->stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    c->ws = static_cast<char*>(workspace_dev);
+    c->L = L;
+    c->shards_loaded = false; c->inited = false; c->num_tiles = 0;
+    c->path = EF21_PATH_AUTO; c->last_path = 0; c->launches = 0;
+    cudaError_t e = cudaMemsetAsync(c->ws + L.status, 0, 256, c->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->x(), 0, (size_t)L.ld * 4, c->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->g(), 0, (size_t)L.ld * 4, c->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->gi(), 0, (size_t)n * L.ld * 4, c->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->msg_idx(), 0, (size_t)n * k * 4, c->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->msg_val(), 0, (size_t)n * k * 4, c->stream);
+    if (e != cudaSuccess) { delete c; return EF21_ERR_CUDA; }
+    *out = c;
+    return EF21_OK;
+}
+
+void ef21_destroy(ef21_ctx* ctx) { delete ctx; }
+
+ef21_status ef21_load_shards(ef21_ctx* c, const float* A_dev, const float* y_dev, const int64_t* row_offsets_host) {
+    if (!c || !row_offsets_host) return EF21_ERR_INVALID_ARG;
+    if (c->N == 0) return EF21_ERR_STATE;
+    if (!A_dev || !y_dev) return EF21_ERR_INVALID_ARG;
+    const unsigned blocks = (unsigned)std::min<i64>(ceil_div(c->N * c->L.ld, 256), 148 * 16);
+    pad_rows_kernel<<<blocks, 256, 0, c->stream>>>(A_dev, c->N, (int)c->d, (int)c->L.ld, c->at<float>(c->L.A));
+    c->launches += 1;
+    CU(cudaGetLastError());
+    CU(cudaMemcpyAsync(c->at<float>(c->L.y), y_dev, (size_t)c->N * 4, cudaMemcpyDeviceToDevice, c->stream));
+    return finish_load(c, reinterpret_cast<const i64*>(row_offsets_host));
+}
+
+ef21_status ef21_load_shards_host(ef21_ctx* c, const float* A_host, const float* y_host, const int64_t* row_offsets_host) {
+    if (!c || !row_offsets_host) return EF21_ERR_INVALID_ARG;
+    if (c->N == 0) return EF21_ERR_STATE;
+    if (!A_host || !y_host) return EF21_ERR_INVALID_ARG;
+    // Host rows have pitch d; the device layout has pitch ld with zero padding.
+    if (c->L.ld != c->d) CU(cudaMemsetAsync(c->at<float>(c->L.A), 0, (size_t)c->N * c->L.ld * 4, c->stream));
+    CU(cudaMemcpy2DAsync(c->at<float>(c->L.A), (size_t)c->L.ld * 4, A_host, (size_t)c->d * 4, (size_t)c->d * 4,
+                         (size_t)c->N, cudaMemcpyHostToDevice, c->stream));
+    CU(cudaMemcpyAsync(c->at<float>(c->L.y), y_host, (size_t)c->N * 4, cudaMemcpyHostToDevice, c->stream));
+    return finish_load(c, reinterpret_cast<const i64*>(row_offsets_host));
+}
+
+ef21_status ef21_set_x(ef21_ctx* c, const float* x0_dev) {
+    if (!c || !x0_dev) return EF21_ERR_INVALID_ARG;
+    CU(cudaMemcpyAsync(c->x(), x0_dev, (size_t)c->d * 4, cudaMemcpyDeviceToDevice, c->stream));
+    return EF21_OK;
+}
+
+ef21_status ef21_init(ef21_ctx* c, int32_t mode) {
+    if (!c || mode < 0 || mode > 2) return EF21_ERR_INVALID_ARG;
+    if (mode == EF21_INIT_ZERO) {
+        EF(zero_state(c));
+        c->inited = true;
+        return EF21_OK;
+    }
+    if (!c->shards_loaded) return EF21_ERR_STATE;
+    EF(enqueue_grads(c, false));
+    return init_from(c, c->at<float>(c->L.grad), c->L.ld, mode);
+}
+
+ef21_status ef21_init_grads(ef21_ctx* c, const float* V_dev, int32_t mode) {
+    if (!c || mode < 0 || mode > 2) return EF21_ERR_INVALID_ARG;
+    if (mode != EF21_INIT_ZERO && !V_dev) return EF21_ERR_INVALID_ARG;
+    return init_from(c, V_dev, c->d, mode);
+}
+
+ef21_status ef21_step(ef21_ctx* c, int32_t steps) {
+    if (!c || steps < 0) return EF21_ERR_INVALID_ARG;
+    if (!c->shards_loaded || !c->inited) return EF21_ERR_STATE;
+    if (c->path == EF21_PATH_PERSISTENT) return EF21_ERR_UNSUPPORTED;
+    for (int t = 0; t < steps; ++t) {
+        EF(enqueue_x_update(c));
+        EF(enqueue_grads(c, false));
+        EF(enqueue_round(c, c->at<float>(c->L.grad), c->L.ld, false));
+    }
+    c->last_path = EF21_PATH_LAUNCHES;
+    return EF21_OK;
+}
+
+ef21_status ef21_step_grads(ef21_ctx* c, const float* V_dev, int32_t steps) {
+    if (!c || !V_dev || steps < 0) return EF21_ERR_INVALID_ARG;
+    if (!c->inited) return EF21_ERR_STATE;
+    for (int t = 0; t < steps; ++t) EF(enqueue_round(c, V_dev, c->d, true));
+    c->last_path = EF21_PATH_LAUNCHES;
+    return EF21_OK;
+}
+
+ef21_status ef21_local_grads(ef21_ctx* c, float* grads_out_dev) {
+    if (!c || !grads_out_dev) return EF21_ERR_INVALID_ARG;
+    if (!c->shards_loaded) return EF21_ERR_STATE;
+    EF(enqueue_grads(c, false));
+    CU(cudaMemcpy2DAsync(grads_out_dev, (size_t)c->d * 4, c->at<float>(c->L.grad), (size_t)c->L.ld * 4,
+                         (size_t)c->d * 4, (size_t)c->n, cudaMemcpyDeviceToDevice, c->stream));
+    return EF21_OK;
+}
+
+size_t ef21_topk_workspace_bytes(int32_t batch, int64_t d, int32_t k) {
+    if (batch < 1 || !valid_shape(1, d, k, 0)) return 0;
+    return topk_layout(batch, d).total;
+}
+
+ef21_status ef21_topk(const float* v_dev, int32_t batch, int64_t d, int32_t k, int32_t* idx_out_dev,
+                      float* val_out_dev, void* workspace_dev, size_t workspace_bytes, void* cuda_stream) {
+    if (!v_dev || !idx_out_dev || !val_out_dev || batch < 1 || batch > 65535 || !valid_shape(1, d, k, 0))
+        return EF21_ERR_INVALID_ARG;
+    TopkLayout L = topk_layout(batch, d);
+    if (!workspace_dev || workspace_bytes < L.total || (reinterpret_cast<uintptr_t>(workspace_dev) % ALIGN) != 0)
+        return EF21_ERR_WORKSPACE;
+    TopkBuffers B = topk_buffers(static_cast<char*>(workspace_dev), L);
+    return enqueue_topk_general(reinterpret_cast<cudaStream_t>(cuda_stream), v_dev, d, nullptr, 0, batch, d, k,
+                                idx_out_dev, val_out_dev, B, nullptr);
+}
+
+static ef21_status copy_state_out(ef21_ctx* c, float* x, float* g, float* gi, int32_t* li, float* lv, cudaMemcpyKind kind) {
+    if (x) CU(cudaMemcpyAsync(x, c->x(), (size_t)c->d * 4, kind, c->stream));
+    if (g) CU(cudaMemcpyAsync(g, c->g(), (size_t)c->d * 4, kind, c->stream));
+    if (gi) CU(cudaMemcpy2DAsync(gi, (size_t)c->d * 4, c->gi(), (size_t)c->L.ld * 4, (size_t)c->d * 4, (size_t)c->n, kind, c->stream));
+    if (li) CU(cudaMemcpyAsync(li, c->msg_idx(), (size_t)c->n * c->k * 4, kind, c->stream));
+    if (lv) CU(cudaMemcpyAsync(lv, c->msg_val(), (size_t)c->n * c->k * 4, kind, c->stream));
+    return EF21_OK;
+}
+
+ef21_status ef21_get_state(ef21_ctx* c, float* x_dev, float* g_dev, float* gi_dev, int32_t* last_idx_dev, float* last_val_dev) {
+    if (!c) return EF21_ERR_INVALID_ARG;
+    return copy_state_out(c, x_dev, g_dev, gi_dev, last_idx_dev, last_val_dev, cudaMemcpyDeviceToDevice);
+}
+
+ef21_status ef21_get_state_host(ef21_ctx* c, float* x_host, float* g_host, float* gi_host, int32_t* last_idx_host, float* last_val_host) {
+    if (!c) return EF21_ERR_INVALID_ARG;
+    EF(copy_state_out(c, x_host, g_host, gi_host, last_idx_host, last_val_host, cudaMemcpyDeviceToHost));
+    CU(cudaStreamSynchronize(c->stream));
+    return EF21_OK;
+}
+
+ef21_status ef21_set_state(ef21_ctx* c, const float* x_dev, const float* g_dev, const float* gi_dev) {
+    if (!c) return EF21_ERR_INVALID_ARG;
+    if (x_dev) CU(cudaMemcpyAsync(c->x(), x_dev, (size_t)c->d * 4, cudaMemcpyDeviceToDevice, c->stream));
+    if (g_dev) CU(cudaMemcpyAsync(c->g(), g_dev, (size_t)c->d * 4, cudaMemcpyDeviceToDevice, c->stream));
+    if (gi_dev) CU(cudaMemcpy2DAsync(c->gi(), (size_t)c->L.ld * 4, gi_dev, (size_t)c->d * 4, (size_t)c->d * 4, (size_t)c->n,
+                                     cudaMemcpyDeviceToDevice, c->stream));
+    c->inited = true;
+    return EF21_OK;
+}
+
+ef21_status ef21_eval(ef21_ctx* c, double* f, double* grad_norm2, double* G) {
+    if (!c) return EF21_ERR_INVALID_ARG;
+    if (!c->shards_loaded) return EF21_ERR_STATE;
+    EF(enqueue_grads(c, true));
+    eval_reduce_kernel<<<1, 1024, 0, c->stream>>>(c->at<double>(c->L.loss_partial), c->at<int>(c->L.tile_begin),
+                                                  c->at<i64>(c->L.row_off), c->at<float>(c->L.grad), c->gi(), c->x(),
+                                                  c->lambda, c->n, (int)c->d, (int)c->L.ld, c->at<double>(c->L.eval_out));
+    c->launches += 1;
+    CU(cudaGetLastError());
+    double out[3];
+    CU(cudaMemcpyAsync(out, c->at<double>(c->L.eval_out), sizeof out, cudaMemcpyDeviceToHost, c->stream));
+    CU(cudaStreamSynchronize(c->stream));
+    if (f) *f = out[0];
+    if (grad_norm2) *grad_norm2 = out[1];
+    if (G) *G = out[2];
+    return EF21_OK;
+}
+
+ef21_status ef21_poll(ef21_ctx* c) {
+    if (!c) return EF21_ERR_INVALID_ARG;
+    unsigned word = 0;
+    CU(cudaMemcpyAsync(&word, c->status(), 4, cudaMemcpyDeviceToHost, c->stream));
+    CU(cudaStreamSynchronize(c->stream));
+    if (word == 0) return EF21_OK;
+    return word <= EF21_ERR_UNSUPPORTED ? (ef21_status)word : EF21_ERR_CUDA;
+}
+
+ef21_status ef21_set_path(ef21_ctx* c, int32_t path) {
+    if (!c || path < EF21_PATH_AUTO || path > EF21_PATH_PERSISTENT) return EF21_ERR_INVALID_ARG;
+    c->path = path;
+    return EF21_OK;
+}
+
+int32_t ef21_last_path(const ef21_ctx* c) { return c ? c->last_path : 0; }
+int64_t ef21_launch_count(const ef21_ctx* c) { return c ? c->launches : 0; }
+
+}  // extern "C"

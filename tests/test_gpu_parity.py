@@ -1,0 +1,273 @@
+"""GPU parity: libef21 (through its C ABI) against the CPU oracle on the same seeded inputs.
+
+Bars: Top-k index sets and values bit-exact given identical input vectors; every state update
+after the gradient bit-exact given identical gradients; local gradients within 1e-5 (relative,
+norm-wise) of the oracle's fp64 gradients per step; x and f(x) within 1e-4 relative after T
+iterations.
+"""
+import numpy as np
+import pytest
+import torch
+
+import ef21_inputs as inputs
+import oracle as oracle_mod
+from gpu_util import (assert_state_bitwise, dev, lockstep, make_gpu, make_oracle_state, rel_l2,
+                      set_gpu_state_from_oracle)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2106_05203_b200 import binding
+    return binding
+
+
+# ---------------------------------------------------------------------------
+# Standalone Top-k
+# ---------------------------------------------------------------------------
+
+def _topk_cases():
+    rng = np.random.default_rng(2024)
+    cases = []
+    for d, k in [(1, 1), (5, 5), (64, 4), (112, 1), (300, 16), (1000, 999), (4096, 1), (4097, 33),
+                 (10007, 10), (70001, 700), (262144, 262), (300000, 299999)]:
+        v = rng.standard_normal(d).astype(np.float32)
+        cases.append((f"gauss-{d}-{k}", v, k))
+    v = inputs.stress_vector(4, 1, 1 << 20)
+    cases.append(("student-1m", v, (1 << 20) // 1000))
+    v = rng.standard_normal(50000).astype(np.float32)
+    v[rng.integers(0, 50000, 20000)] = np.float32(-0.75)            # many exact ties around the cut
+    cases.append(("ties", v, 25000))
+    cases.append(("all-equal", np.full(9000, 2.5, dtype=np.float32), 1234))
+    cases.append(("all-zero", np.zeros(5000, dtype=np.float32), 7))
+    v = np.zeros(6000, dtype=np.float32); v[[17, 4000, 5999]] = [1.0, -2.0, 3.0]; v[5] = -0.0
+    cases.append(("fewer-nonzeros-than-k", v, 10))
+    v = (rng.integers(-3, 4, 33333)).astype(np.float32) * np.float32(0.5)   # few distinct magnitudes
+    cases.append(("quantised", v, 11111))
+    v = rng.standard_normal(8192).astype(np.float32) * np.float32(1e-41)     # subnormals
+    cases.append(("subnormal", v, 100))
+    return cases
+
+
+@pytest.mark.parametrize("name,v,k", _topk_cases(), ids=[c[0] for c in _topk_cases()])
+def test_topk_bit_exact(name, v, k, B, oracle32):
+    idx, val = B.topk(dev(v), k)
+    oi, ov = oracle32.topk(v, k)
+    np.testing.assert_array_equal(idx.cpu().numpy()[0], oi)
+    np.testing.assert_array_equal(val.cpu().numpy()[0].view(np.uint32), ov.view(np.uint32))
+
+
+def test_topk_batch_and_repeatability(B, oracle32):
+    V = np.stack([inputs.stress_vector(7, i, 50001) for i in range(5)])
+    idx, val = B.topk(dev(V), 50)
+    idx2, val2 = B.topk(dev(V), 50)
+    assert torch.equal(idx, idx2) and torch.equal(val, val2)
+    for i in range(5):
+        oi, ov = oracle32.topk(V[i], 50)
+        np.testing.assert_array_equal(idx[i].cpu().numpy(), oi)
+        np.testing.assert_array_equal(val[i].cpu().numpy(), ov)
+
+
+# ---------------------------------------------------------------------------
+# Local gradients (Eq. 19)
+# ---------------------------------------------------------------------------
+
+@pytest.mark.parametrize("cfg", [0, 1, 2, 3])
+def test_local_gradients_within_1e5(cfg, B, oracle32):
+    w = inputs.config(cfg)
+    h = make_gpu(w)
+    rng = np.random.default_rng(cfg)
+    for x in (w.x0, (rng.standard_normal(w.d) * 0.3).astype(np.float32)):
+        h.set_x(dev(x))
+        got = h.local_grads().cpu().numpy()
+        want = oracle32.all_grads(w.A, w.y, w.row_offsets, x, w.lam)
+        for i in range(w.n):
+            assert rel_l2(got[i], want[i]) <= 1e-5, (cfg, i)
+    # at x = 0 with binary features every partial sum is exact: bit-identical gradients
+    if cfg in (1, 2, 3):
+        h.set_x(dev(w.x0))
+        got = h.local_grads().cpu().numpy()
+        want = oracle32.all_grads(w.A, w.y, w.row_offsets, w.x0, w.lam)
+        np.testing.assert_array_equal(got, want)
+
+
+def test_local_gradients_uneven_and_empty_shards(B, oracle32):
+    w = inputs.config(0)
+    w.row_offsets = np.array([0, 0, 3, 150, 200], dtype=np.int64)     # an empty shard and ragged ones
+    h = make_gpu(w)
+    x = np.linspace(-0.5, 0.5, w.d).astype(np.float32)
+    h.set_x(dev(x))
+    got = h.local_grads().cpu().numpy()
+    want = oracle32.all_grads(w.A, w.y, w.row_offsets, x, w.lam)
+    for i in range(w.n):
+        assert rel_l2(got[i], want[i]) <= 1e-5
+
+
+def test_eval_matches_oracle(B, oracle32):
+    w = inputs.config(0)
+    h = make_gpu(w); h.init(B.INIT_COMPRESSED); h.step(5)
+    x, g, gi, _, _ = h.get_state_host()
+    f, nrm2, G = h.eval()
+    assert f == pytest.approx(oracle32.loss(w.A, w.y, w.row_offsets, x, w.lam), rel=1e-6)
+    on, oG = oracle32.diagnostics(w.A, w.y, w.row_offsets, x, w.lam, gi)
+    assert nrm2 == pytest.approx(on, rel=1e-4)
+    assert G == pytest.approx(oG, rel=1e-4)
+
+
+# ---------------------------------------------------------------------------
+# Algorithm 2 with supplied gradients: everything is bit-exact
+# ---------------------------------------------------------------------------
+
+@pytest.mark.parametrize("n,d,k,mode", [(2, 4, 1, 0), (4, 64, 4, 0), (3, 5000, 50, 1), (8, 70001, 70, 0),
+                                        (5, 300, 300, 2), (20, 112, 1, 1), (1, 1, 1, 0), (64, 4097, 4, 1)])
+def test_supplied_gradients_bit_exact(n, d, k, mode, B, oracle32):
+    V = np.stack([inputs.stress_vector(100 + n, i, d) for i in range(n)])
+    gamma = 0.01
+    h = B.EF21(n, d, k, gamma)
+    st = oracle_mod.State(oracle32, n, d, k, gamma)
+    Vd = dev(V)
+    h.init_grads(Vd, mode); st.init_from_grads(V, mode)
+    assert_state_bitwise(h, st, "init")
+    for t in range(6):
+        h.step_grads(Vd, 1); st.step_grads(V, 1)
+        assert_state_bitwise(h, st, f"step {t}")
+    h.step_grads(Vd, 5); st.step_grads(V, 5)
+    assert_state_bitwise(h, st, "5 steps in one call")
+    assert h.poll() == 0
+
+
+def test_hand_worked_example_on_gpu(B):
+    # the same hand-derived run of Algorithm 2 the oracle is pinned to (tests/golden)
+    from test_oracle_pins import _read_hand_example
+    scal, vec = _read_hand_example()
+    V = np.array([vec["V1"], vec["V2"]], dtype=np.float32)
+    h = B.EF21(2, 4, 1, scal["gamma"])
+    h.init_grads(dev(V), 0)
+    for t in range(4):
+        x, g, gi, li, lv = h.get_state_host()
+        np.testing.assert_array_equal(x, vec[(f"t{t}", "x")])
+        np.testing.assert_array_equal(g, vec[(f"t{t}", "g")])
+        np.testing.assert_array_equal(gi[0], vec[(f"t{t}", "g1")])
+        np.testing.assert_array_equal(gi[1], vec[(f"t{t}", "g2")])
+        if t:
+            np.testing.assert_array_equal(li[:, 0], vec[(f"t{t}", "idx")])
+            np.testing.assert_array_equal(lv[:, 0], vec[(f"t{t}", "val")])
+        h.step_grads(dev(V), 1)
+
+
+def test_changing_supplied_gradients(B, oracle32):
+    n, d, k = 6, 3001, 30
+    rng = np.random.default_rng(3)
+    h = B.EF21(n, d, k, 0.05); st = oracle_mod.State(oracle32, n, d, k, 0.05)
+    h.init_grads(None, 1); st.init(1)
+    for t in range(8):
+        V = rng.standard_normal((n, d)).astype(np.float32)
+        h.step_grads(dev(V), 1); st.step_grads(V, 1)
+        assert_state_bitwise(h, st, f"step {t}")
+
+
+# ---------------------------------------------------------------------------
+# Algorithm 2 on the logistic objective
+# ---------------------------------------------------------------------------
+
+@pytest.mark.parametrize("mode", [0, 1, 2])
+def test_init_modes(mode, B, oracle32):
+    w = inputs.config(1)
+    h = make_gpu(w); st = make_oracle_state(oracle32, w)
+    h.init(mode); st.init(mode)
+    if mode == 0:
+        assert_state_bitwise(h, st, "init mode 0")
+    x, g, gi, _, _ = h.get_state_host()
+    np.testing.assert_array_equal(gi, st.gi)      # x0 = 0 and binary features: exact
+    np.testing.assert_array_equal(g, st.g)
+
+
+def test_teacher_forced_steps_tiny(B, oracle32):
+    w = inputs.config(0)
+    h = make_gpu(w); st = make_oracle_state(oracle32, w)
+    h.init(0); st.init(0)
+    set_gpu_state_from_oracle(h, st)
+    for t in range(20):
+        st_prev_gi = st.gi.copy()
+        h.step(1); st.step(1)
+        x, g, gi, li, lv = h.get_state_host()
+        np.testing.assert_array_equal(x, st.x)                    # x update is exact given g
+        np.testing.assert_array_equal(li, st.idx)
+        assert np.max(np.abs(lv - st.val)) <= 1e-5 * np.max(np.abs(st.val))
+        set_gpu_state_from_oracle(h, st)
+
+
+def test_free_running_tiny_T100(B, oracle32):
+    w = inputs.config(0)
+    h = make_gpu(w); st = make_oracle_state(oracle32, w)
+    h.init(0); st.init(0)
+    h.step(w.T); st.step(w.T)
+    x, g, gi, _, _ = h.get_state_host()
+    assert rel_l2(x, st.x) <= 1e-4
+    assert rel_l2(g, st.g) <= 1e-3
+    f_gpu = h.eval()[0]
+    assert f_gpu == pytest.approx(st.loss(), rel=1e-4)
+    assert oracle32.loss(w.A, w.y, w.row_offsets, x, w.lam) == pytest.approx(st.loss(), rel=1e-4)
+    assert h.poll() == 0
+
+
+@pytest.mark.parametrize("cfg,k,steps", [(1, 1, 150), (2, 1, 40), (2, 4, 40), (2, 16, 40), (3, 1, 25)])
+def test_lockstep_paper_shapes(cfg, k, steps, B, oracle32):
+    w = inputs.config(cfg, k=k)
+    h = make_gpu(w, k=k); st = make_oracle_state(oracle32, w, k=k)
+    h.init(0); st.init(0)
+    assert_state_bitwise(h, st, "init")
+    rebased = lockstep(h, st, oracle32, w, steps, k=k)
+    assert rebased <= max(2, steps // 10)
+    x = h.get_state_host()[0]
+    assert rel_l2(x, st.x) <= 1e-4
+
+
+def test_k_equals_d_is_gradient_descent_on_gpu(B, oracle32):
+    # Section 5.2: EF21 with k = d is GD; g_i tracks grad f_i to a few ulps in fp32.
+    w = inputs.config(0, k=64)
+    h = make_gpu(w, k=64)
+    h.init(0); h.step(10)
+    x, g, gi, _, _ = h.get_state_host()
+    grads = h.local_grads().cpu().numpy()
+    assert np.max(np.abs(gi - grads)) <= 8 * np.finfo(np.float32).eps * np.max(np.abs(grads))
+    np.testing.assert_allclose(g, gi.astype(np.float64).mean(axis=0), rtol=0, atol=1e-6)
+
+
+def test_bitwise_reproducible_and_resume(B):
+    w = inputs.config(2, k=4)
+    runs = []
+    for _ in range(2):
+        h = make_gpu(w, k=4); h.init(0); h.step(30)
+        runs.append(h.get_state_host())
+    for a, b in zip(runs[0], runs[1]):
+        np.testing.assert_array_equal(a, b)
+    # checkpoint / resume: 15 steps, copy the state into a fresh handle, 15 more
+    h1 = make_gpu(w, k=4); h1.init(0); h1.step(15)
+    x, g, gi, _, _ = h1.get_state()
+    h2 = make_gpu(w, k=4); h2.set_state(x, g, gi); h2.step(15)
+    for a, b in zip(h2.get_state_host(messages=False)[:3], runs[0][:3]):
+        np.testing.assert_array_equal(a, b)
+
+
+def test_call_order_and_argument_errors(B):
+    w = inputs.config(0)
+    h = B.EF21(w.n, w.d, w.k, w.gamma, w.lam, total_rows=w.N)
+    with pytest.raises(B.Ef21Error) as e:
+        h.step(1)
+    assert e.value.status == 2
+    with pytest.raises(B.Ef21Error) as e:
+        h.init(0)                       # shards not loaded
+    assert e.value.status == 2
+    bad = w.row_offsets.copy(); bad[-1] -= 1
+    with pytest.raises(B.Ef21Error) as e:
+        h.load_shards(dev(w.A), dev(w.y), bad)
+    assert e.value.status == 1
+    h.load_shards(dev(w.A), dev(w.y), w.row_offsets)
+    with pytest.raises(B.Ef21Error):
+        h.step(1)                       # not initialised
+    h.init(1); h.step(1)
+    assert h.poll() == 0
+    with pytest.raises(B.Ef21Error):
+        B.EF21(4, 64, 65, 0.1)          # k > d
