@@ -151,6 +151,25 @@ ef21_status ef21_eval(ef21_ctx* ctx, double* f, double* grad_norm2, double* G);
  * error a kernel recorded (EF21_ERR_TIMEOUT, EF21_ERR_NONFINITE), or EF21_ERR_CUDA. */
 ef21_status ef21_poll(ef21_ctx* ctx);
 
+/* Clears the device status word (after an error has been read with ef21_poll). */
+ef21_status ef21_clear_status(ef21_ctx* ctx);
+
+/* Self-check of the bounded device-side wait used by the persistent path: one thread spins
+ * at most spin_limit (1 .. 2^24) times on a word that nothing writes, then records
+ * EF21_ERR_TIMEOUT, which the next ef21_poll returns.  The device and the context stay usable. */
+ef21_status ef21_selftest_bounded_wait(ef21_ctx* ctx, uint32_t spin_limit);
+
+/* Tuning of the persistent path (Algorithm 2 as one kernel; worker i = one thread-block
+ * cluster): blocks per cluster (1..8, 0 = automatic), rows per warp batch (8, 16, 32, 0 =
+ * automatic) and where the shard rows live (0 registers, 1 shared memory, 2 global memory /
+ * L2, -1 = automatic).  A shape that cannot run makes ef21_step fall back (path AUTO) or
+ * return EF21_ERR_UNSUPPORTED (path PERSISTENT).  get_ reports what the last persistent
+ * launch used. */
+ef21_status ef21_set_persistent_shape(ef21_ctx* ctx, int32_t cluster_blocks, int32_t rows_per_batch,
+                                      int32_t row_source);
+ef21_status ef21_get_persistent_shape(const ef21_ctx* ctx, int32_t* cluster_blocks,
+                                      int32_t* rows_per_batch, int32_t* row_source);
+
 /* Forces an execution path (EF21_PATH_*) for later ef21_step calls. */
 ef21_status ef21_set_path(ef21_ctx* ctx, int32_t path);
 /* The path the last ef21_step / ef21_step_grads actually used (EF21_PATH_*), 0 if none yet. */

@@ -46,6 +46,10 @@ SIGNATURES = {
     "ef21_set_state": (ctypes.c_int, [_vp, _vp, _vp, _vp]),
     "ef21_eval": (ctypes.c_int, [_vp, _dp, _dp, _dp]),
     "ef21_poll": (ctypes.c_int, [_vp]),
+    "ef21_clear_status": (ctypes.c_int, [_vp]),
+    "ef21_selftest_bounded_wait": (ctypes.c_int, [_vp, ctypes.c_uint32]),
+    "ef21_set_persistent_shape": (ctypes.c_int, [_vp, _i32, _i32, _i32]),
+    "ef21_get_persistent_shape": (ctypes.c_int, [_vp, ctypes.POINTER(_i32), ctypes.POINTER(_i32), ctypes.POINTER(_i32)]),
     "ef21_set_path": (ctypes.c_int, [_vp, _i32]),
     "ef21_last_path": (_i32, [_vp]),
     "ef21_launch_count": (_i64, [_vp]),
@@ -220,6 +224,22 @@ class EF21:
 
     def poll(self) -> int:
         return int(_lib.ef21_poll(self._h))
+
+    def clear_status(self) -> None:
+        _check(_lib.ef21_clear_status(self._h), "ef21_clear_status")
+
+    def selftest_bounded_wait(self, spin_limit: int) -> None:
+        _check(_lib.ef21_selftest_bounded_wait(self._h, spin_limit), "ef21_selftest_bounded_wait")
+
+    def set_persistent_shape(self, cluster_blocks: int = 0, rows_per_batch: int = 0, row_source: int = -1) -> None:
+        _check(_lib.ef21_set_persistent_shape(self._h, cluster_blocks, rows_per_batch, row_source),
+               "ef21_set_persistent_shape")
+
+    def get_persistent_shape(self):
+        c, r, s = _i32(), _i32(), _i32()
+        _check(_lib.ef21_get_persistent_shape(self._h, ctypes.byref(c), ctypes.byref(r), ctypes.byref(s)),
+               "ef21_get_persistent_shape")
+        return c.value, r.value, s.value
 
     def set_path(self, path: int) -> None:
         _check(_lib.ef21_set_path(self._h, path), "ef21_set_path")

@@ -10,6 +10,7 @@
 #include "apply.cuh"
 #include "common.cuh"
 #include "grad.cuh"
+#include "persistent.cuh"
 #include "topk.cuh"
 
 using namespace ef21;
@@ -54,7 +55,7 @@ struct Layout {
     int agg_tiles;     // tiles of AGG_TILE coordinates
     int tile_rows;     // rows per gradient tile
     i64 max_tiles;     // capacity of the gradient tile table
-    size_t status, x, g, gi, msg_idx, msg_val, topk, agg_off, eval_out;
+    size_t status, x, g, gi, msg_idx, msg_val, topk, agg_off, eval_out, slots;
     size_t A, y, row_off, tile_begin, tiles, partial, loss_partial, grad;
     size_t total;
     TopkLayout tk;
@@ -76,6 +77,7 @@ Layout make_layout(i64 n, i64 d, i64 k, i64 N) {
     L.topk = take(L.tk.total);
     L.agg_off = take((size_t)n * (L.agg_tiles + 1) * 4);
     L.eval_out = take(256);
+    L.slots = take((size_t)2 * n * k * 8);
     L.tile_rows = 0; L.max_tiles = 0;
     L.A = L.y = L.row_off = L.tile_begin = L.tiles = L.partial = L.loss_partial = L.grad = 0;
     if (N > 0) {
@@ -108,6 +110,9 @@ struct ef21_ctx {
     bool shards_loaded, inited;
     int num_tiles;
     int path, last_path;
+    int pk_cluster, pk_rb, pk_src;      // forced persistent-kernel shape (0 / -1 = automatic)
+    int pk_used_cluster, pk_used_rb, pk_used_src;
+    unsigned spin_limit;
     i64 launches;
     std::vector<i64> row_off;
     std::vector<RowTile> tiles;
@@ -269,6 +274,135 @@ ef21_status finish_load(ef21_ctx* c, const i64* row_offsets_host) {
     return EF21_OK;
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Persistent path
+// ---------------------------------------------------------------------------------------------
+
+typedef void (*PersistKernel)(const PersistParams);
+
+template <int CHUNKS, int RB>
+PersistKernel pk_by_src(int src) {
+    if (src == PK_SRC_REG) return persistent_kernel<CHUNKS, RB, PK_SRC_REG>;
+    if (src == PK_SRC_SMEM) return persistent_kernel<CHUNKS, RB, PK_SRC_SMEM>;
+    return persistent_kernel<CHUNKS, RB, PK_SRC_GMEM>;
+}
+
+PersistKernel pk_lookup(int chunks, int rb, int src) {
+    switch (chunks * 100 + rb) {
+        case 108: return pk_by_src<1, 8>(src);
+        case 116: return pk_by_src<1, 16>(src);
+        case 132: return pk_by_src<1, 32>(src);
+        case 208: return pk_by_src<2, 8>(src);
+        case 216: return pk_by_src<2, 16>(src);
+        case 308: return pk_by_src<3, 8>(src);
+        case 408: return pk_by_src<4, 8>(src);
+    }
+    return nullptr;
+}
+
+struct PersistPlan {
+    bool ok;
+    int C, rb, src, chunks;
+    size_t smem;
+    PersistKernel kernel;
+};
+
+size_t pk_smem_bytes(int ld, int C, int nmsg, int src, i64 rows_cta) {
+    size_t b = (size_t)(5 + PK_WARPS + C) * ld * 4 + (size_t)((nmsg + 1) & ~1) * 8;
+    if (src == PK_SRC_SMEM) b += (size_t)rows_cta * ld * 4;
+    return b;
+}
+
+// Chooses cluster size, rows per batch and the source of the shard rows; checks that all n
+// clusters can be resident at once (the blocks wait on one another through global memory).
+PersistPlan plan_persistent(ef21_ctx* c) {
+    PersistPlan P; P.ok = false;
+    const int ld = (int)c->L.ld;
+    if (!c->shards_loaded || ld > 512 || c->k > PK_MAX_K || (i64)c->n * c->k > PK_MAX_MSGS) return P;
+    int dev = 0, sms = 0, max_smem = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return P;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    const int chunk_slots = (ld / 4 + 31) / 32;
+    const int max_rb = chunk_slots == 1 ? 32 : (chunk_slots == 2 ? 16 : 8);
+    i64 max_m = 0;
+    for (int i = 0; i < c->n; ++i) max_m = std::max<i64>(max_m, c->row_off[i + 1] - c->row_off[i]);
+    const int nmsg = c->n * c->k;
+    for (int C = 8; C >= 1; --C) {
+        if (c->pk_cluster > 0 && C != c->pk_cluster) continue;
+        if ((i64)c->n * C > sms) continue;
+        const i64 rows_cta = ceil_div(std::max<i64>(max_m, 1), C);
+        if (c->pk_cluster == 0 && C > 1 && rows_cta < 8) continue;       // do not split below one batch
+        int rb = 0, src = PK_SRC_GMEM;
+        for (int cand = 8; cand <= max_rb; cand *= 2)
+            if (ceil_div(rows_cta, cand) <= PK_WARPS) { rb = cand; src = PK_SRC_REG; break; }
+        if (rb == 0) {
+            rb = max_rb;
+            src = pk_smem_bytes(ld, C, nmsg, PK_SRC_SMEM, rows_cta) <= (size_t)max_smem - 1024 ? PK_SRC_SMEM : PK_SRC_GMEM;
+        }
+        if (c->pk_rb > 0) {
+            if (c->pk_rb > max_rb) continue;
+            rb = c->pk_rb;
+            if (src == PK_SRC_REG && ceil_div(rows_cta, rb) > PK_WARPS) src = PK_SRC_SMEM;
+        }
+        if (c->pk_src >= 0) {
+            if (c->pk_src == PK_SRC_REG && ceil_div(rows_cta, rb) > PK_WARPS) continue;
+            src = c->pk_src;
+        }
+        const size_t smem = pk_smem_bytes(ld, C, nmsg, src, rows_cta);
+        if (smem > (size_t)max_smem - 1024) continue;
+        PersistKernel kern = pk_lookup(chunk_slots, rb, src);
+        if (!kern) continue;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+            cudaGetLastError();
+            continue;
+        }
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(c->n * C)); cfg.blockDim = dim3(PK_THREADS); cfg.dynamicSmemBytes = smem;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)C; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        int active = 0;
+        if (cudaOccupancyMaxActiveClusters(&active, kern, &cfg) != cudaSuccess) { cudaGetLastError(); continue; }
+        if (active < c->n) continue;
+        P.ok = true; P.C = C; P.rb = rb; P.src = src; P.chunks = chunk_slots; P.smem = smem; P.kernel = kern;
+        return P;
+    }
+    return P;
+}
+
+ef21_status run_persistent(ef21_ctx* c, const PersistPlan& P, int steps) {
+    PersistParams p;
+    p.A = c->at<float>(c->L.A); p.y = c->at<float>(c->L.y); p.row_off = c->at<i64>(c->L.row_off);
+    p.x = c->x(); p.g = c->g(); p.gi = c->gi(); p.msg_idx = c->msg_idx(); p.msg_val = c->msg_val();
+    p.slots = c->at<unsigned long long>(c->L.slots); p.status = c->status();
+    p.n = c->n; p.d = (int)c->d; p.ld = (int)c->L.ld; p.k = c->k; p.C = P.C; p.steps = steps;
+    p.slice_rows = 0; p.gamma = c->gamma; p.lambda = c->lambda; p.inv_n = 1.0f / (float)c->n;
+    p.spin_limit = c->spin_limit; p.epoch0 = 0u;
+    CU(cudaMemsetAsync(p.slots, 0, (size_t)2 * c->n * c->k * 8, c->stream));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(c->n * P.C)); cfg.blockDim = dim3(PK_THREADS); cfg.dynamicSmemBytes = P.smem;
+    cfg.stream = c->stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)P.C; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeCooperative;
+    attr[1].val.cooperative = 1;
+    cfg.attrs = attr; cfg.numAttrs = 2;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, P.kernel, p);
+    if (e != cudaSuccess) {           // residency was already checked; retry as a plain cluster launch
+        cudaGetLastError();
+        cfg.numAttrs = 1;
+        e = cudaLaunchKernelEx(&cfg, P.kernel, p);
+    }
+    if (e != cudaSuccess) { cudaGetLastError(); return EF21_ERR_CUDA; }
+    c->launches += 1;
+    c->pk_used_cluster = P.C; c->pk_used_rb = P.rb; c->pk_used_src = P.src;
+    return EF21_OK;
+}
+
 }  // namespace
 
 // ---------------------------------------------------------------------------------------------
@@ -311,6 +445,9 @@ ef21_status ef21_create(ef21_ctx** out, int32_t n, int64_t d, int32_t k, float g
     c->L = L;
     c->shards_loaded = false; c->inited = false; c->num_tiles = 0;
     c->path = EF21_PATH_AUTO; c->last_path = 0; c->launches = 0;
+    c->pk_cluster = 0; c->pk_rb = 0; c->pk_src = -1;
+    c->pk_used_cluster = c->pk_used_rb = 0; c->pk_used_src = -1;
+    c->spin_limit = 1u << 22;
     cudaError_t e = cudaMemsetAsync(c->ws + L.status, 0, 256, c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->x(), 0, (size_t)L.ld * 4, c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->g(), 0, (size_t)L.ld * 4, c->stream);
@@ -375,7 +512,16 @@ ef21_status ef21_init_grads(ef21_ctx* c, const float* V_dev, int32_t mode) {
 ef21_status ef21_step(ef21_ctx* c, int32_t steps) {
     if (!c || steps < 0) return EF21_ERR_INVALID_ARG;
     if (!c->shards_loaded || !c->inited) return EF21_ERR_STATE;
-    if (c->path == EF21_PATH_PERSISTENT) return EF21_ERR_UNSUPPORTED;
+    if (steps == 0) return EF21_OK;
+    if (c->path != EF21_PATH_LAUNCHES) {
+        PersistPlan P = plan_persistent(c);
+        if (P.ok) {
+            EF(run_persistent(c, P, steps));
+            c->last_path = EF21_PATH_PERSISTENT;
+            return EF21_OK;
+        }
+        if (c->path == EF21_PATH_PERSISTENT) return EF21_ERR_UNSUPPORTED;
+    }
     for (int t = 0; t < steps; ++t) {
         EF(enqueue_x_update(c));
         EF(enqueue_grads(c, false));
@@ -480,6 +626,37 @@ ef21_status ef21_poll(ef21_ctx* c) {
 ef21_status ef21_set_path(ef21_ctx* c, int32_t path) {
     if (!c || path < EF21_PATH_AUTO || path > EF21_PATH_PERSISTENT) return EF21_ERR_INVALID_ARG;
     c->path = path;
+    return EF21_OK;
+}
+
+ef21_status ef21_set_persistent_shape(ef21_ctx* c, int32_t cluster_blocks, int32_t rows_per_batch, int32_t row_source) {
+    if (!c || cluster_blocks < 0 || cluster_blocks > 8) return EF21_ERR_INVALID_ARG;
+    if (rows_per_batch != 0 && rows_per_batch != 8 && rows_per_batch != 16 && rows_per_batch != 32) return EF21_ERR_INVALID_ARG;
+    if (row_source < -1 || row_source > 2) return EF21_ERR_INVALID_ARG;
+    c->pk_cluster = cluster_blocks; c->pk_rb = rows_per_batch; c->pk_src = row_source;
+    return EF21_OK;
+}
+
+ef21_status ef21_get_persistent_shape(const ef21_ctx* c, int32_t* cluster_blocks, int32_t* rows_per_batch, int32_t* row_source) {
+    if (!c) return EF21_ERR_INVALID_ARG;
+    if (cluster_blocks) *cluster_blocks = c->pk_used_cluster;
+    if (rows_per_batch) *rows_per_batch = c->pk_used_rb;
+    if (row_source) *row_source = c->pk_used_src;
+    return EF21_OK;
+}
+
+ef21_status ef21_clear_status(ef21_ctx* c) {
+    if (!c) return EF21_ERR_INVALID_ARG;
+    CU(cudaMemsetAsync(c->status(), 0, 256, c->stream));
+    return EF21_OK;
+}
+
+ef21_status ef21_selftest_bounded_wait(ef21_ctx* c, uint32_t spin_limit) {
+    if (!c || spin_limit == 0 || spin_limit > (1u << 24)) return EF21_ERR_INVALID_ARG;
+    CU(cudaMemsetAsync(c->at<unsigned long long>(c->L.slots), 0, 8, c->stream));
+    bounded_wait_selftest_kernel<<<1, 1, 0, c->stream>>>(c->at<unsigned long long>(c->L.slots), c->status(), spin_limit);
+    c->launches += 1;
+    CU(cudaGetLastError());
     return EF21_OK;
 }
 

@@ -1,0 +1,354 @@
+// EF21 (Algorithm 2) as ONE persistent kernel for small dimensions (d <= 512, k <= 32):
+// all `steps` iterations run inside a single launch, the shards stay on chip.
+//
+// Mapping.  Worker i is a thread-block cluster of C blocks; block c of the cluster owns a
+// contiguous slice of the worker's rows, held in registers (REG), in shared memory (SMEM) or
+// re-read from global memory / L2 every iteration (GMEM).  Every block keeps its own replica of
+// x and g, so the only grid-wide dependency per iteration is the exchange of the n messages
+// c_i (k pairs each), which plays the role of the paper's "send c_i to the master / broadcast x":
+//
+//   1. x <- fma(-gamma, g, x)                                   (every block, its replica)
+//   2. rows in batches of RB per warp: margins a_r.x by a transposed warp reduction (lane L ends
+//      up with the margin of row L/(32/RB)), residual rho_r, rank-1 accumulation rho_r a_r
+//   3. block partial -> leader block of the cluster through distributed shared memory
+//   4. leader block: grad_i = sum/m_i + regulariser' and v = grad_i - g_i, one coordinate per
+//      thread; its warp 0 then takes Top-k by k rounds of a warp arg-max on (|v| bits, lower index
+//      wins), updates g_i += c_i and publishes k packed 64-bit words (epoch:16 | index:16 |
+//      value bits:32) into a double-buffered global slot array
+//   5. every block polls the n*k words of this iteration's epoch (bounded spin), then each
+//      coordinate thread adds the matching values in ascending worker order: g += (1/n) sum c_i
+//
+// All summation orders are fixed by the launch shape, so two runs give identical bits.  A wait
+// that exceeds its spin limit records EF21_ERR_TIMEOUT in the status word; from then on every
+// block skips work but keeps arriving at the cluster barriers, so the kernel always terminates.
+#pragma once
+#include <cooperative_groups.h>
+
+#include "common.cuh"
+
+namespace ef21 {
+namespace cg = cooperative_groups;
+
+constexpr int PK_THREADS = 256;
+constexpr int PK_WARPS = PK_THREADS / 32;
+constexpr int PK_MAX_K = 32;
+constexpr int PK_MAX_MSGS = 2048;       // n*k words staged in shared memory
+enum { PK_SRC_REG = 0, PK_SRC_SMEM = 1, PK_SRC_GMEM = 2 };
+
+struct PersistParams {
+    const float* A;            // [N][ld], padded, read-only
+    const float* y;            // [N]
+    const i64* row_off;        // [n+1]
+    float* x;                  // [ld]
+    float* g;                  // [ld]
+    float* gi;                 // [n][ld]
+    int* msg_idx;              // [n][k] last messages (written at the final iteration)
+    float* msg_val;
+    unsigned long long* slots; // [2][n*k]
+    unsigned* status;
+    int n, d, ld, k, C, steps;
+    int slice_rows;            // capacity (rows) of the shared-memory slice (SMEM source)
+    float gamma, lambda, inv_n;
+    unsigned spin_limit;
+    unsigned epoch0;           // epoch of the first iteration minus one
+};
+
+__device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_relaxed_u64(unsigned long long* p, unsigned long long v) {
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ unsigned ld_relaxed_u32(const unsigned* p) {
+    unsigned v;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// Sum of v[r] over the 32 lanes for RB rows at once: after the call lane L holds the total of
+// row L / (32/RB).  RB-1 shuffles for the halving steps plus log2(32/RB) butterfly steps.
+template <int RB>
+__device__ __forceinline__ float reduce_rows(float (&v)[RB], int lane) {
+#pragma unroll
+    for (int half = RB / 2, off = 16; half >= 1; half >>= 1, off >>= 1) {
+        const bool upper = (lane & off) != 0;
+#pragma unroll
+        for (int r = 0; r < half; ++r) {
+            const float keep = upper ? v[r + half] : v[r];
+            const float send = upper ? v[r] : v[r + half];
+            v[r] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+        }
+    }
+    float s = v[0];
+#pragma unroll
+    for (int off = (32 / RB) / 2; off >= 1; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+    return s;
+}
+
+__device__ __forceinline__ float4 fma4(float s, float4 a, float4 c) {
+    c.x = fmaf(s, a.x, c.x); c.y = fmaf(s, a.y, c.y); c.z = fmaf(s, a.z, c.z); c.w = fmaf(s, a.w, c.w);
+    return c;
+}
+__device__ __forceinline__ float dot4(float4 a, float4 b, float z) {
+    z = fmaf(a.x, b.x, z); z = fmaf(a.y, b.y, z); z = fmaf(a.z, b.z, z); z = fmaf(a.w, b.w, z);
+    return z;
+}
+__device__ __forceinline__ float comp_of(const float4& v, int c) {
+    return c == 0 ? v.x : (c == 1 ? v.y : (c == 2 ? v.z : v.w));
+}
+
+template <int CHUNKS, int RB, int SRC>
+__global__ void __launch_bounds__(PK_THREADS, 1) persistent_kernel(const PersistParams p) {
+    constexpr int SH = (RB == 32) ? 0 : (RB == 16 ? 1 : 2);    // log2(32/RB)
+    static_assert(RB == 8 || RB == 16 || RB == 32, "RB");
+    static_assert(RB * CHUNKS <= 32, "register budget");
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    cg::cluster_group cluster = cg::this_cluster();
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int C = p.C, ld = p.ld, chunks = ld >> 2;
+    const int crank = (int)cluster.block_rank();
+    const int worker = blockIdx.x / C;
+    const int nmsg = p.n * p.k;
+
+    // ---- shared memory carve-up -------------------------------------------------------------
+    float* xs = reinterpret_cast<float*>(smem_raw);                 // [ld]
+    float* gs = xs + ld;                                            // [ld]
+    float* rterm = gs + ld;                                         // [ld] regulariser term at x
+    float* gis = rterm + ld;                                        // [ld] g_i (leader block)
+    float* vs = gis + ld;                                           // [ld] v = grad_i - g_i (leader block)
+    float* red = vs + ld;                                           // [PK_WARPS][ld]
+    float* part = red + PK_WARPS * ld;                              // [C][ld] (used in the leader)
+    unsigned long long* msg = reinterpret_cast<unsigned long long*>(part + C * ld);   // [nmsg]
+    float* slice = reinterpret_cast<float*>(msg + ((nmsg + 1) & ~1));                  // SMEM source
+    __shared__ int abort_flag;
+
+    // ---- this block's rows --------------------------------------------------------------------
+    const i64 w_r0 = p.row_off[worker], w_r1 = p.row_off[worker + 1];
+    const i64 m_i = w_r1 - w_r0;
+    const i64 q = (m_i + C - 1) / C;
+    const i64 r0 = min(w_r0 + (i64)crank * q, w_r1), r1 = min(r0 + q, w_r1);
+    const int rows = (int)(r1 - r0);
+    const int nbatch = (rows + RB - 1) / RB;
+
+    if (tid == 0) abort_flag = 0;
+    for (int j = tid; j < ld; j += PK_THREADS) { xs[j] = p.x[j]; gs[j] = p.g[j]; }
+    if (SRC == PK_SRC_SMEM) {
+        const float4* src = reinterpret_cast<const float4*>(p.A + r0 * (i64)ld);
+        float4* dst = reinterpret_cast<float4*>(slice);
+        for (int e = tid; e < rows * chunks; e += PK_THREADS) dst[e] = src[e];
+    }
+
+    // The leader block of the cluster keeps g_i in shared memory.
+    const bool leader = crank == 0;
+    if (leader)
+        for (int j = tid; j < ld; j += PK_THREADS) gis[j] = p.gi[(i64)worker * ld + j];
+
+    // REG source: the (single) batch of this warp lives in registers for the whole kernel.
+    float4 a[RB][CHUNKS];
+    float y_reg = 0.f;
+    auto load_batch = [&](int b) {
+        const int rb0 = b * RB;
+#pragma unroll
+        for (int r = 0; r < RB; ++r) {
+            const int row = rb0 + r;
+#pragma unroll
+            for (int cs = 0; cs < CHUNKS; ++cs) {
+                const int c = lane + 32 * cs;
+                float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (row < rows && c < chunks) {
+                    if (SRC == PK_SRC_SMEM) v = reinterpret_cast<const float4*>(slice)[row * chunks + c];
+                    else v = __ldg(reinterpret_cast<const float4*>(p.A + (r0 + row) * (i64)ld) + c);
+                }
+                a[r][cs] = v;
+            }
+        }
+        const int myrow = rb0 + (lane >> SH);
+        y_reg = myrow < rows ? __ldg(p.y + r0 + myrow) : 0.f;
+    };
+    if (SRC == PK_SRC_REG) load_batch(warp);     // host guarantees nbatch <= PK_WARPS
+    __syncthreads();
+
+    bool aborted = false;
+    for (int t = 0; t < p.steps; ++t) {
+        const unsigned epoch = (p.epoch0 + (unsigned)t + 1u) & 0xffffu;
+        unsigned long long* slot = p.slots + (size_t)(epoch & 1u) * nmsg;
+
+        if (!aborted) {
+            // 1. x <- x - gamma g on this block's replica (Algorithm 2, first line of the loop)
+            for (int j = tid; j < ld; j += PK_THREADS) {
+                const float xj = fmaf(-p.gamma, gs[j], xs[j]);
+                xs[j] = xj;
+                rterm[j] = regulariser_grad(p.lambda, xj);
+            }
+            __syncthreads();
+
+            // 2. partial gradient over this warp's batches
+            float4 xr[CHUNKS], acc[CHUNKS];
+#pragma unroll
+            for (int cs = 0; cs < CHUNKS; ++cs) {
+                const int c = lane + 32 * cs;
+                xr[cs] = c < chunks ? reinterpret_cast<const float4*>(xs)[c] : make_float4(0.f, 0.f, 0.f, 0.f);
+                acc[cs] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            for (int b = warp; b < nbatch; b += PK_WARPS) {
+                if (SRC != PK_SRC_REG) load_batch(b);
+                float pd[RB];
+#pragma unroll
+                for (int r = 0; r < RB; ++r) {
+                    float z = 0.f;
+#pragma unroll
+                    for (int cs = 0; cs < CHUNKS; ++cs) z = dot4(a[r][cs], xr[cs], z);
+                    pd[r] = z;
+                }
+                const float z = reduce_rows<RB>(pd, lane);
+                const float rho = logistic_residual(y_reg, z);
+#pragma unroll
+                for (int r = 0; r < RB; ++r) {
+                    const float pr = __shfl_sync(0xffffffffu, rho, r << SH);
+#pragma unroll
+                    for (int cs = 0; cs < CHUNKS; ++cs) acc[cs] = fma4(pr, a[r][cs], acc[cs]);
+                }
+            }
+#pragma unroll
+            for (int cs = 0; cs < CHUNKS; ++cs) {
+                const int c = lane + 32 * cs;
+                if (c < chunks) reinterpret_cast<float4*>(red + warp * ld)[c] = acc[cs];
+            }
+            __syncthreads();
+
+            // 3. block partial (warps in ascending order) -> leader's shared memory
+            float* leader_part = C > 1 ? cluster.map_shared_rank(part, 0) : part;
+            for (int j = tid; j < ld; j += PK_THREADS) {
+                float s = red[j];
+#pragma unroll
+                for (int w = 1; w < PK_WARPS; ++w) s = __fadd_rn(s, red[w * ld + j]);
+                leader_part[crank * ld + j] = s;
+            }
+        }
+        if (C > 1) cluster.sync(); else __syncthreads();
+
+        if (!aborted) {
+            // 4. leader: gradient, difference, Top-k, state update, publish
+            if (leader) {
+                const float mf = (float)m_i;
+                for (int j = tid; j < ld; j += PK_THREADS) {
+                    float sum = part[j];
+                    for (int cc = 1; cc < C; ++cc) sum = __fadd_rn(sum, part[cc * ld + j]);
+                    const float grad = __fadd_rn(m_i > 0 ? __fdiv_rn(sum, mf) : 0.f, rterm[j]);
+                    vs[j] = __fsub_rn(grad, gis[j]);
+                }
+                __syncthreads();
+            }
+            if (leader && warp == 0) {
+                float4 v[CHUNKS];
+                unsigned taken = 0u;                  // bit (cs*4+comp) set: not selectable
+#pragma unroll
+                for (int cs = 0; cs < CHUNKS; ++cs) {
+                    const int c = lane + 32 * cs;
+                    v[cs] = c < chunks ? reinterpret_cast<const float4*>(vs)[c] : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        if (4 * c + e >= p.d) taken |= 1u << (cs * 4 + e);
+                }
+                int my_idx = 0; float my_val = 0.f;          // lane t keeps the t-th pick
+                for (int t2 = 0; t2 < p.k; ++t2) {
+                    long long best = -1;
+#pragma unroll
+                    for (int cs = 0; cs < CHUNKS; ++cs)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const unsigned idx = (unsigned)(4 * (lane + 32 * cs) + e);
+                            const long long comp = ((long long)mag_key(comp_of(v[cs], e)) << 32) | (long long)(0xffffffffu - idx);
+                            const bool ok = !((taken >> (cs * 4 + e)) & 1u);
+                            best = (ok && comp > best) ? comp : best;
+                        }
+#pragma unroll
+                    for (int off = 16; off >= 1; off >>= 1) {
+                        const long long o = __shfl_xor_sync(0xffffffffu, best, off);
+                        best = o > best ? o : best;
+                    }
+                    const unsigned widx = 0xffffffffu - (unsigned)(best & 0xffffffffll);
+                    const int wchunk = (int)(widx >> 2), wlane = wchunk & 31, wcs = wchunk >> 5, we = (int)(widx & 3u);
+                    float wval = 0.f;
+#pragma unroll
+                    for (int cs = 0; cs < CHUNKS; ++cs)
+                        if (cs == wcs) wval = comp_of(v[cs], we);
+                    wval = __shfl_sync(0xffffffffu, wval, wlane);
+                    if (lane == wlane) {
+                        taken |= 1u << (wcs * 4 + we);
+                        gis[widx] = __fadd_rn(gis[widx], wval);
+                    }
+                    if (lane == t2) { my_idx = (int)widx; my_val = wval; }
+                }
+                // ascending index order inside the message
+                int rank = 0;
+                for (int u = 0; u < p.k; ++u) {
+                    const int oi = __shfl_sync(0xffffffffu, my_idx, u);
+                    rank += (lane < p.k && oi < my_idx) ? 1 : 0;
+                }
+                if (lane < p.k) {
+                    const unsigned long long word = ((unsigned long long)epoch << 48) |
+                                                    ((unsigned long long)(unsigned)my_idx << 32) |
+                                                    (unsigned long long)__float_as_uint(my_val);
+                    st_relaxed_u64(slot + worker * p.k + rank, word);
+                    if (t == p.steps - 1) {
+                        p.msg_idx[worker * p.k + rank] = my_idx;
+                        p.msg_val[worker * p.k + rank] = my_val;
+                    }
+                }
+            }
+
+            // 5. gather all n*k message words of this epoch (bounded spin)
+            for (int u = tid; u < nmsg; u += PK_THREADS) {
+                unsigned spins = 0;
+                unsigned long long w;
+                while (true) {
+                    w = ld_relaxed_u64(slot + u);
+                    if ((unsigned)(w >> 48) == epoch) break;
+                    ++spins;
+                    if ((spins & 1023u) == 0u && ld_relaxed_u32(p.status) != 0u) { abort_flag = 1; break; }
+                    if (spins > p.spin_limit) { record_error(p.status, (unsigned)5 /* EF21_ERR_TIMEOUT */); abort_flag = 1; break; }
+                }
+                msg[u] = w;
+            }
+            __syncthreads();
+            if (abort_flag) aborted = true;
+        }
+        if (!aborted) {
+            // g_j += (1/n) * sum over workers (ascending) of the values sent for coordinate j
+            for (int j = tid; j < p.d; j += PK_THREADS) {
+                float s = 0.f; bool touched = false;
+#pragma unroll 4
+                for (int u = 0; u < nmsg; ++u) {
+                    const unsigned long long w = msg[u];
+                    if ((int)((w >> 32) & 0xffffu) == j) { s = __fadd_rn(s, __uint_as_float((unsigned)w)); touched = true; }
+                }
+                if (touched) gs[j] = __fadd_rn(gs[j], __fmul_rn(s, p.inv_n));
+            }
+            // the next iteration's x update reads gs[j] in the same thread: no barrier needed here
+        }
+    }
+
+    __syncthreads();
+    if (blockIdx.x == 0)
+        for (int j = tid; j < ld; j += PK_THREADS) { p.x[j] = xs[j]; p.g[j] = gs[j]; }
+    if (leader)
+        for (int j = tid; j < ld; j += PK_THREADS) p.gi[(i64)worker * ld + j] = gis[j];
+}
+
+// One-block self-check of the bounded wait: spins on a word that nobody writes and must come back
+// with EF21_ERR_TIMEOUT in the status word instead of hanging.
+__global__ void bounded_wait_selftest_kernel(const unsigned long long* never_written, unsigned* status,
+                                             unsigned spin_limit) {
+    unsigned spins = 0;
+    while (true) {
+        const unsigned long long w = ld_relaxed_u64(never_written);
+        if ((unsigned)(w >> 48) == 0xffffu) break;
+        if (++spins > spin_limit) { record_error(status, 5u); break; }
+    }
+}
+
+}  // namespace ef21
