@@ -151,6 +151,15 @@ ef21_status ef21_eval(ef21_ctx* ctx, double* f, double* grad_norm2, double* G);
  * error a kernel recorded (EF21_ERR_TIMEOUT, EF21_ERR_NONFINITE), or EF21_ERR_CUDA. */
 ef21_status ef21_poll(ef21_ctx* ctx);
 
+/* Top-k algorithm used inside the EF21 rounds of the launch path: 0 = automatic (long vectors,
+ * d >= 2^18 and k <= 8192, take the one-pass path: sampled threshold, single streaming pass,
+ * exact selection among the candidates; everything else takes the multi-pass radix select),
+ * 1 = always the multi-pass radix select.  Both give the same bits. */
+ef21_status ef21_set_topk_algorithm(ef21_ctx* ctx, int32_t algorithm);
+/* Number of vectors, since creation, for which the one-pass Top-k had to fall back to the exact
+ * selection over the whole vector (threshold missed or too many ties); synchronises. */
+ef21_status ef21_fallback_count(ef21_ctx* ctx, int64_t* count);
+
 /* Clears the device status word (after an error has been read with ef21_poll). */
 ef21_status ef21_clear_status(ef21_ctx* ctx);
 

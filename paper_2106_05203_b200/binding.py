@@ -46,6 +46,8 @@ SIGNATURES = {
     "ef21_set_state": (ctypes.c_int, [_vp, _vp, _vp, _vp]),
     "ef21_eval": (ctypes.c_int, [_vp, _dp, _dp, _dp]),
     "ef21_poll": (ctypes.c_int, [_vp]),
+    "ef21_set_topk_algorithm": (ctypes.c_int, [_vp, _i32]),
+    "ef21_fallback_count": (ctypes.c_int, [_vp, ctypes.POINTER(_i64)]),
     "ef21_clear_status": (ctypes.c_int, [_vp]),
     "ef21_selftest_bounded_wait": (ctypes.c_int, [_vp, ctypes.c_uint32]),
     "ef21_set_persistent_shape": (ctypes.c_int, [_vp, _i32, _i32, _i32]),
@@ -224,6 +226,14 @@ class EF21:
 
     def poll(self) -> int:
         return int(_lib.ef21_poll(self._h))
+
+    def set_topk_algorithm(self, algorithm: int) -> None:
+        _check(_lib.ef21_set_topk_algorithm(self._h, algorithm), "ef21_set_topk_algorithm")
+
+    def fallback_count(self) -> int:
+        v = _i64()
+        _check(_lib.ef21_fallback_count(self._h, ctypes.byref(v)), "ef21_fallback_count")
+        return int(v.value)
 
     def clear_status(self) -> None:
         _check(_lib.ef21_clear_status(self._h), "ef21_clear_status")

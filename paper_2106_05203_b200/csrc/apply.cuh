@@ -76,6 +76,86 @@ aggregate_kernel(const int* __restrict__ idx, const float* __restrict__ val, con
     }
 }
 
+// The same aggregation with the tile's message entries first staged in shared memory (one
+// parallel gather), so that the ordered pass over the workers touches shared memory only.
+// Needs n <= AGG_STAGE_MAX_N; a tile with more than AGG_STAGE_CAP entries takes the direct loop.
+constexpr int AGG_STAGE_MAX_N = 1024;
+constexpr int AGG_STAGE_CAP = 3072;
+
+template <bool UPDATE_X>
+__global__ void __launch_bounds__(AGG_BLOCK)
+aggregate_staged_kernel(const int* __restrict__ idx, const float* __restrict__ val, const int* __restrict__ off,
+                        int n, int k, int ntiles, i64 d, float inv_n, float gamma,
+                        float* __restrict__ g, float* __restrict__ x) {
+    __shared__ float s[AGG_TILE];
+    __shared__ unsigned char touched[AGG_TILE];
+    __shared__ int w_start[AGG_STAGE_MAX_N + 1];
+    __shared__ int w_lo[AGG_STAGE_MAX_N];
+    __shared__ unsigned short e_idx[AGG_STAGE_CAP];
+    __shared__ float e_val[AGG_STAGE_CAP];
+    __shared__ unsigned scratch[33];
+    const int b = blockIdx.x;
+    const i64 j0 = (i64)b * AGG_TILE;
+    for (int t = threadIdx.x; t < AGG_TILE; t += AGG_BLOCK) { s[t] = 0.f; touched[t] = 0; }
+    unsigned base = 0u;
+    for (int c0 = 0; c0 < n; c0 += AGG_BLOCK) {
+        const int i = c0 + threadIdx.x;
+        int lo = 0, hi = 0;
+        if (i < n) { lo = off[(i64)i * (ntiles + 1) + b]; hi = off[(i64)i * (ntiles + 1) + b + 1]; }
+        unsigned tot;
+        const unsigned pre = block_excl_scan((unsigned)(hi - lo), scratch, tot);
+        if (i < n) { w_start[i] = (int)(base + pre); w_lo[i] = lo; }
+        base += tot;
+    }
+    if (threadIdx.x == 0) w_start[n] = (int)base;
+    __syncthreads();
+    const int total = (int)base;
+    if (total <= AGG_STAGE_CAP) {
+        for (int e = threadIdx.x; e < total; e += AGG_BLOCK) {
+            int lo = 0, hi = n;                      // last worker i with w_start[i] <= e
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (w_start[mid] <= e) lo = mid; else hi = mid;
+            }
+            const i64 src = (i64)lo * k + w_lo[lo] + (e - w_start[lo]);
+            e_idx[e] = (unsigned short)((i64)idx[src] - j0);
+            e_val[e] = val[src];
+        }
+        __syncthreads();
+        for (int i = 0; i < n; ++i) {
+            const int lo = w_start[i], hi = w_start[i + 1];
+            if (lo == hi) continue;                  // uniform: read from shared memory
+            for (int e = lo + threadIdx.x; e < hi; e += AGG_BLOCK) {
+                const int t = e_idx[e];
+                s[t] = __fadd_rn(s[t], e_val[e]);
+                touched[t] = 1;
+            }
+            __syncthreads();
+        }
+    } else {
+        for (int i = 0; i < n; ++i) {
+            const int lo = w_lo[i], hi = lo + (w_start[i + 1] - w_start[i]);
+            for (int e = lo + threadIdx.x; e < hi; e += AGG_BLOCK) {
+                const int t = (int)((i64)idx[(i64)i * k + e] - j0);
+                s[t] = __fadd_rn(s[t], val[(i64)i * k + e]);
+                touched[t] = 1;
+            }
+            __syncthreads();
+        }
+    }
+    for (int t = threadIdx.x; t < AGG_TILE; t += AGG_BLOCK) {
+        const i64 j = j0 + t;
+        if (j >= d) break;
+        if (UPDATE_X) {
+            const float gj = g[j];
+            x[j] = fmaf(-gamma, gj, x[j]);
+            if (touched[t]) g[j] = __fadd_rn(gj, __fmul_rn(s[t], inv_n));
+        } else if (touched[t]) {
+            g[j] = __fadd_rn(g[j], __fmul_rn(s[t], inv_n));
+        }
+    }
+}
+
 // x <- fma(-gamma, g, x), elementwise.
 __global__ void x_update_kernel(const float* __restrict__ g, float* __restrict__ x, i64 d, float gamma) {
     for (i64 j = blockIdx.x * (i64)blockDim.x + threadIdx.x; j < d; j += (i64)gridDim.x * blockDim.x)

@@ -11,6 +11,7 @@
 #include "common.cuh"
 #include "grad.cuh"
 #include "persistent.cuh"
+#include "stress.cuh"
 #include "topk.cuh"
 
 using namespace ef21;
@@ -28,15 +29,31 @@ inline i64 ceil_div(i64 a, i64 b) { return (a + b - 1) / b; }
 struct TopkLayout {
     size_t state, hist, chunks, total;
     int nchunks;
+    // one-pass path for long vectors (stress.cuh); fast == false: sections absent
+    bool fast;
+    int nreg;
+    size_t thr, flags, slow_count, region_cnt, cand;
 };
 
-TopkLayout topk_layout(i64 batch, i64 d) {
+bool fast_topk_eligible(i64 d, i64 k) { return d >= ST_MIN_D && k <= ST_MAX_K; }
+
+TopkLayout topk_layout(i64 batch, i64 d, i64 k) {
     TopkLayout L;
     L.nchunks = (int)ceil_div(d, TK_CHUNK);
     size_t o = 0;
     L.state = o; o += align_up((size_t)batch * sizeof(TkState));
     L.hist = o; o += align_up((size_t)batch * TK_BINS * sizeof(unsigned));
     L.chunks = o; o += align_up((size_t)batch * (size_t)L.nchunks * sizeof(uint2));
+    L.fast = fast_topk_eligible(d, k);
+    L.nreg = (int)ceil_div(d, ST_SUB);
+    L.thr = L.flags = L.slow_count = L.region_cnt = L.cand = 0;
+    if (L.fast) {
+        L.thr = o; o += align_up((size_t)batch * 4);
+        L.flags = o; o += align_up((size_t)batch * 4);
+        L.slow_count = o; o += align_up(4);
+        L.region_cnt = o; o += align_up((size_t)batch * L.nreg * 4);
+        L.cand = o; o += align_up((size_t)batch * L.nreg * ST_REGION_CAP * sizeof(int2));
+    }
     L.total = o;
     return L;
 }
@@ -65,7 +82,7 @@ Layout make_layout(i64 n, i64 d, i64 k, i64 N) {
     Layout L;
     L.ld = (d + 3) / 4 * 4;
     L.agg_tiles = (int)ceil_div(d, AGG_TILE);
-    L.tk = topk_layout(n, d);
+    L.tk = topk_layout(n, d, k);
     size_t o = 0;
     auto take = [&](size_t bytes) { size_t at = o; o += align_up(bytes); return at; };
     L.status = take(256);
@@ -113,6 +130,7 @@ struct ef21_ctx {
     int pk_cluster, pk_rb, pk_src;      // forced persistent-kernel shape (0 / -1 = automatic)
     int pk_used_cluster, pk_used_rb, pk_used_src;
     unsigned spin_limit;
+    bool force_general_topk;
     i64 launches;
     std::vector<i64> row_off;
     std::vector<RowTile> tiles;
@@ -142,6 +160,8 @@ namespace {
 
 struct TopkBuffers {
     TkState* state; unsigned* hist; uint2* chunks; int nchunks;
+    bool fast; int nreg;
+    unsigned* thr; unsigned* flags; unsigned* slow_count; int* region_cnt; int2* cand;
 };
 
 TopkBuffers topk_buffers(char* base, const TopkLayout& L) {
@@ -150,7 +170,45 @@ TopkBuffers topk_buffers(char* base, const TopkLayout& L) {
     B.hist = reinterpret_cast<unsigned*>(base + L.hist);
     B.chunks = reinterpret_cast<uint2*>(base + L.chunks);
     B.nchunks = L.nchunks;
+    B.fast = L.fast; B.nreg = L.nreg;
+    B.thr = reinterpret_cast<unsigned*>(base + L.thr);
+    B.flags = reinterpret_cast<unsigned*>(base + L.flags);
+    B.slow_count = reinterpret_cast<unsigned*>(base + L.slow_count);
+    B.region_cnt = reinterpret_cast<int*>(base + L.region_cnt);
+    B.cand = reinterpret_cast<int2*>(base + L.cand);
     return B;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Exact Top-k of v = a - b for long vectors in one pass over a and b (see stress.cuh).  If gi_rows
+// is given, g_i += c_i is applied by the same kernel that writes the messages.
+ef21_status enqueue_topk_fast(cudaStream_t st, const float* a, i64 pitch_a, const float* b, i64 pitch_b,
+                              int batch, i64 d, int k, int* idx_out, float* val_out, float* gi_rows, i64 ld,
+                              const TopkBuffers& B, i64* launches) {
+    static bool smem_set = false;
+    const size_t finish_smem = (size_t)ST_CAND_CAP * 8 + 2048 * 4;
+    if (!smem_set) {
+        CU(cudaFuncSetAttribute(st_finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)finish_smem));
+        smem_set = true;
+    }
+    const i64 target = std::max<i64>(2 * (i64)k, (i64)k + 2048);
+    i64 rank = ceil_div(target * (i64)(ST_SAMPLE_BLOCKS * ST_SAMPLE_LEN), d);
+    rank = std::min<i64>(std::max<i64>(rank, 32), ST_SAMPLE_BLOCKS * ST_SAMPLE_LEN / 2);
+    st_sample_kernel<<<batch, ST_THREADS, 0, st>>>(a, pitch_a, b, pitch_b, d, (unsigned)rank, B.thr, B.flags);
+    dim3 grid((unsigned)ceil_div(B.nreg, ST_COLLECT_WARPS), (unsigned)batch);
+    const bool vec = aligned16(a) && pitch_a % 4 == 0 && (!b || (aligned16(b) && pitch_b % 4 == 0));
+    if (vec)
+        st_collect_kernel<true><<<grid, ST_COLLECT_WARPS * 32, 0, st>>>(a, pitch_a, b, pitch_b, d, B.nreg, B.thr, B.cand,
+                                                                        B.region_cnt, B.flags);
+    else
+        st_collect_kernel<false><<<grid, ST_COLLECT_WARPS * 32, 0, st>>>(a, pitch_a, b, pitch_b, d, B.nreg, B.thr, B.cand,
+                                                                         B.region_cnt, B.flags);
+    st_finish_kernel<<<batch, ST_THREADS, finish_smem, st>>>(a, pitch_a, b, pitch_b, d, B.nreg, k, B.cand, B.region_cnt,
+                                                             B.flags, idx_out, val_out, gi_rows, ld, B.slow_count);
+    if (launches) *launches += 3;
+    CU(cudaGetLastError());
+    return EF21_OK;
 }
 
 // Exact Top-k of v = a - b for `batch` vectors (b may be null); general multi-block path.
@@ -192,24 +250,27 @@ ef21_status enqueue_grads(ef21_ctx* c, bool with_loss) {
 // x <- x - gamma g_old fused into the aggregation).
 ef21_status enqueue_round(ef21_ctx* c, const float* a, i64 pitch_a, bool update_x) {
     TopkBuffers B = topk_buffers(c->ws + c->L.topk, c->L.tk);
-    EF(enqueue_topk_general(c->stream, a, pitch_a, c->gi(), c->L.ld, c->n, c->d, c->k, c->msg_idx(),
-                            c->msg_val(), B, &c->launches));
-    const i64 total = (i64)c->n * c->k;
-    apply_messages_kernel<<<(unsigned)ceil_div(total, 256), 256, 0, c->stream>>>(c->msg_idx(), c->msg_val(), total,
-                                                                                c->k, c->L.ld, c->gi());
+    if (B.fast && !c->force_general_topk) {
+        EF(enqueue_topk_fast(c->stream, a, pitch_a, c->gi(), c->L.ld, c->n, c->d, c->k, c->msg_idx(), c->msg_val(),
+                             c->gi(), c->L.ld, B, &c->launches));
+    } else {
+        EF(enqueue_topk_general(c->stream, a, pitch_a, c->gi(), c->L.ld, c->n, c->d, c->k, c->msg_idx(),
+                                c->msg_val(), B, &c->launches));
+        const i64 total = (i64)c->n * c->k;
+        apply_messages_kernel<<<(unsigned)ceil_div(total, 256), 256, 0, c->stream>>>(c->msg_idx(), c->msg_val(), total,
+                                                                                    c->k, c->L.ld, c->gi());
+        c->launches += 1;
+    }
     const i64 noff = (i64)c->n * (c->L.agg_tiles + 1);
     agg_offsets_kernel<<<(unsigned)ceil_div(noff, 256), 256, 0, c->stream>>>(c->msg_idx(), c->n, c->k,
                                                                             c->L.agg_tiles, c->at<int>(c->L.agg_off));
     const float inv_n = 1.0f / (float)c->n;
-    if (update_x)
-        aggregate_kernel<true><<<c->L.agg_tiles, AGG_BLOCK, 0, c->stream>>>(
-            c->msg_idx(), c->msg_val(), c->at<int>(c->L.agg_off), c->n, c->k, c->L.agg_tiles, c->d, inv_n,
-            c->gamma, c->g(), c->x());
-    else
-        aggregate_kernel<false><<<c->L.agg_tiles, AGG_BLOCK, 0, c->stream>>>(
-            c->msg_idx(), c->msg_val(), c->at<int>(c->L.agg_off), c->n, c->k, c->L.agg_tiles, c->d, inv_n,
-            c->gamma, c->g(), c->x());
-    c->launches += 3;
+    auto kern = c->n <= AGG_STAGE_MAX_N
+                    ? (update_x ? aggregate_staged_kernel<true> : aggregate_staged_kernel<false>)
+                    : (update_x ? aggregate_kernel<true> : aggregate_kernel<false>);
+    kern<<<c->L.agg_tiles, AGG_BLOCK, 0, c->stream>>>(c->msg_idx(), c->msg_val(), c->at<int>(c->L.agg_off), c->n, c->k,
+                                                      c->L.agg_tiles, c->d, inv_n, c->gamma, c->g(), c->x());
+    c->launches += 2;
     CU(cudaGetLastError());
     return EF21_OK;
 }
@@ -448,12 +509,14 @@ ef21_status ef21_create(ef21_ctx** out, int32_t n, int64_t d, int32_t k, float g
     c->pk_cluster = 0; c->pk_rb = 0; c->pk_src = -1;
     c->pk_used_cluster = c->pk_used_rb = 0; c->pk_used_src = -1;
     c->spin_limit = 1u << 22;
+    c->force_general_topk = false;
     cudaError_t e = cudaMemsetAsync(c->ws + L.status, 0, 256, c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->x(), 0, (size_t)L.ld * 4, c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->g(), 0, (size_t)L.ld * 4, c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->gi(), 0, (size_t)n * L.ld * 4, c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->msg_idx(), 0, (size_t)n * k * 4, c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->msg_val(), 0, (size_t)n * k * 4, c->stream);
+    if (e == cudaSuccess && L.tk.fast) e = cudaMemsetAsync(c->ws + L.topk + L.tk.slow_count, 0, 4, c->stream);
     if (e != cudaSuccess) { delete c; return EF21_ERR_CUDA; }
     *out = c;
     return EF21_OK;
@@ -549,20 +612,22 @@ ef21_status ef21_local_grads(ef21_ctx* c, float* grads_out_dev) {
 }
 
 size_t ef21_topk_workspace_bytes(int32_t batch, int64_t d, int32_t k) {
-    if (batch < 1 || !valid_shape(1, d, k, 0)) return 0;
-    return topk_layout(batch, d).total;
+    if (batch < 1 || batch > 65535 || !valid_shape(1, d, k, 0)) return 0;
+    return topk_layout(batch, d, k).total;
 }
 
 ef21_status ef21_topk(const float* v_dev, int32_t batch, int64_t d, int32_t k, int32_t* idx_out_dev,
                       float* val_out_dev, void* workspace_dev, size_t workspace_bytes, void* cuda_stream) {
     if (!v_dev || !idx_out_dev || !val_out_dev || batch < 1 || batch > 65535 || !valid_shape(1, d, k, 0))
         return EF21_ERR_INVALID_ARG;
-    TopkLayout L = topk_layout(batch, d);
+    TopkLayout L = topk_layout(batch, d, k);
     if (!workspace_dev || workspace_bytes < L.total || (reinterpret_cast<uintptr_t>(workspace_dev) % ALIGN) != 0)
         return EF21_ERR_WORKSPACE;
     TopkBuffers B = topk_buffers(static_cast<char*>(workspace_dev), L);
-    return enqueue_topk_general(reinterpret_cast<cudaStream_t>(cuda_stream), v_dev, d, nullptr, 0, batch, d, k,
-                                idx_out_dev, val_out_dev, B, nullptr);
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    if (B.fast)
+        return enqueue_topk_fast(st, v_dev, d, nullptr, 0, batch, d, k, idx_out_dev, val_out_dev, nullptr, 0, B, nullptr);
+    return enqueue_topk_general(st, v_dev, d, nullptr, 0, batch, d, k, idx_out_dev, val_out_dev, B, nullptr);
 }
 
 static ef21_status copy_state_out(ef21_ctx* c, float* x, float* g, float* gi, int32_t* li, float* lv, cudaMemcpyKind kind) {
@@ -642,6 +707,23 @@ ef21_status ef21_get_persistent_shape(const ef21_ctx* c, int32_t* cluster_blocks
     if (cluster_blocks) *cluster_blocks = c->pk_used_cluster;
     if (rows_per_batch) *rows_per_batch = c->pk_used_rb;
     if (row_source) *row_source = c->pk_used_src;
+    return EF21_OK;
+}
+
+ef21_status ef21_set_topk_algorithm(ef21_ctx* c, int32_t algorithm) {
+    if (!c || algorithm < 0 || algorithm > 1) return EF21_ERR_INVALID_ARG;
+    c->force_general_topk = algorithm == 1;
+    return EF21_OK;
+}
+
+ef21_status ef21_fallback_count(ef21_ctx* c, int64_t* count) {
+    if (!c || !count) return EF21_ERR_INVALID_ARG;
+    unsigned v = 0;
+    if (c->L.tk.fast) {
+        CU(cudaMemcpyAsync(&v, c->ws + c->L.topk + c->L.tk.slow_count, 4, cudaMemcpyDeviceToHost, c->stream));
+        CU(cudaStreamSynchronize(c->stream));
+    }
+    *count = (int64_t)v;
     return EF21_OK;
 }
 
