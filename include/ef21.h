@@ -134,6 +134,30 @@ ef21_status ef21_topk(const float* v_dev, int32_t batch, int64_t d, int32_t k,
                       int32_t* idx_out_dev, float* val_out_dev,
                       void* workspace_dev, size_t workspace_bytes, void* cuda_stream);
 
+/* Top-k for callers that cannot hand over or allocate device scratch.  (The paper has no
+ * counterpart: this is a packaging variant of ef21_topk, same result bit for bit.)
+ *
+ * Who needs it: code that runs where the CUDA allocator is off limits -- a host thread that may
+ * not block on the implicit synchronisation of cudaMalloc/cudaFree, a plug-in inside a framework
+ * that owns all device memory and hands out none, a process whose memory was carved up at start
+ * and must not grow.  Such a caller passes only its input and the two output arrays; the
+ * scratch is a fixed 1 MiB array inside the library image (every GPU that loads the library
+ * holds it until the process exits).  The function calls no cudaMalloc, cudaFree or allocating
+ * library routine.
+ *
+ * Limits: batch <= 64 and batch * ceil(d / 4096) <= 16384 (e.g. 64 vectors of 2^20 entries, or
+ * one of 2^26); beyond that the call returns EF21_ERR_UNSUPPORTED and does nothing.  Always
+ * runs the multi-pass radix select.
+ * The first call on a device looks up the device address of the scratch array
+ * (cudaGetSymbolAddress, with that device current) and caches it; make that first call outside
+ * of any stream capture.
+ * All calls in a process share the one scratch array, which keeps the previous call's contents:
+ * every call clears what it needs at zero on the stream before use.  Two calls whose kernels can
+ * overlap on the GPU (different streams without an ordering between them) race on it; order
+ * them.  Arguments as for ef21_topk. */
+ef21_status ef21_topk_static(const float* v_dev, int32_t batch, int64_t d, int32_t k,
+                             int32_t* idx_out_dev, float* val_out_dev, void* cuda_stream);
+
 /* Copies of the state; any pointer may be NULL.  gi is [n][d]; last_idx/last_val are the
  * most recent messages c_i, [n][k] each.  set_state also marks the handle initialised
  * (resume / teacher forcing); x, g or gi left NULL keep their current contents. */

@@ -41,6 +41,7 @@ SIGNATURES = {
     "ef21_local_grads": (ctypes.c_int, [_vp, _vp]),
     "ef21_topk_workspace_bytes": (_sz, [_i32, _i64, _i32]),
     "ef21_topk": (ctypes.c_int, [_vp, _i32, _i64, _i32, _vp, _vp, _vp, _sz, _vp]),
+    "ef21_topk_static": (ctypes.c_int, [_vp, _i32, _i64, _i32, _vp, _vp, _vp]),
     "ef21_get_state": (ctypes.c_int, [_vp, _vp, _vp, _vp, _vp, _vp]),
     "ef21_get_state_host": (ctypes.c_int, [_vp, _vp, _vp, _vp, _vp, _vp]),
     "ef21_set_state": (ctypes.c_int, [_vp, _vp, _vp, _vp]),
@@ -281,3 +282,22 @@ def topk(v: torch.Tensor, k: int, stream: Optional[torch.cuda.Stream] = None):
                               _stream_handle(stream)), "ef21_topk")
         ws.record_stream(stream if stream is not None else torch.cuda.current_stream())
     return idx, val
+
+
+def topk_static(v: torch.Tensor, k: int, idx: torch.Tensor, val: torch.Tensor,
+                stream: Optional[torch.cuda.Stream] = None) -> None:
+    """ef21_topk_static: Top-k into caller-provided outputs idx[batch, k] (int32) and val[batch, k]
+    (float32) with no device scratch handed over and none allocated; for callers that must not
+    touch the CUDA allocator.  Raises Ef21Error(EF21_ERR_UNSUPPORTED) beyond the built-in scratch
+    (batch <= 64, batch * ceil(d / 4096) <= 16384)."""
+    if v.dim() == 1:
+        v = v.unsqueeze(0)
+    _dev_f32(v)
+    batch, d = v.shape
+    if not (idx.is_cuda and idx.dtype == torch.int32 and idx.is_contiguous() and idx.numel() == batch * k):
+        raise TypeError("idx must be a contiguous int32 CUDA tensor with batch*k entries")
+    if not (val.is_cuda and val.dtype == torch.float32 and val.is_contiguous() and val.numel() == batch * k):
+        raise TypeError("val must be a contiguous float32 CUDA tensor with batch*k entries")
+    with torch.cuda.device(v.device):
+        _check(_lib.ef21_topk_static(_ptr(v), batch, d, k, _ptr(idx), _ptr(val), _stream_handle(stream)),
+               "ef21_topk_static")

@@ -4,6 +4,7 @@
 #include <cmath>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -628,6 +629,60 @@ ef21_status ef21_topk(const float* v_dev, int32_t batch, int64_t d, int32_t k, i
     if (B.fast)
         return enqueue_topk_fast(st, v_dev, d, nullptr, 0, batch, d, k, idx_out_dev, val_out_dev, nullptr, 0, B, nullptr);
     return enqueue_topk_general(st, v_dev, d, nullptr, 0, batch, d, k, idx_out_dev, val_out_dev, B, nullptr);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Top-k without any caller-provided or allocated scratch
+// ---------------------------------------------------------------------------------------------
+// Scratch of ef21_topk_static: lives in the library image, so every GPU that loads the library
+// holds these bytes until the process exits.
+constexpr size_t TOPK_STATIC_SCRATCH_BYTES = (size_t)1 << 20;
+constexpr int TOPK_STATIC_MAX_BATCH = 64;
+constexpr i64 TOPK_STATIC_MAX_CHUNKS = 16384;      // batch * ceil(d / 4096)
+static __device__ __align__(256) unsigned char g_topk_static_scratch[TOPK_STATIC_SCRATCH_BYTES];
+
+// Device address of the scratch array on the current device.  In host code the array's name is only
+// a handle for the runtime, not an address a kernel could use, so the address is asked for once
+// per device (with that device current) and cached.
+static ef21_status topk_static_scratch(void** out) {
+    constexpr int MAX_DEVICES = 64;
+    static std::mutex mu;
+    static void* addr[MAX_DEVICES] = {};
+    int dev = -1;
+    CU(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= MAX_DEVICES) return EF21_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!addr[dev]) {
+        void* p = nullptr;
+        CU(cudaGetSymbolAddress(&p, g_topk_static_scratch));
+        if (!p) return EF21_ERR_CUDA;
+        addr[dev] = p;
+    }
+    *out = addr[dev];
+    return EF21_OK;
+}
+
+ef21_status ef21_topk_static(const float* v_dev, int32_t batch, int64_t d, int32_t k, int32_t* idx_out_dev,
+                             float* val_out_dev, void* cuda_stream) {
+    if (!v_dev || !idx_out_dev || !val_out_dev || batch < 1 || !valid_shape(1, d, k, 0)) return EF21_ERR_INVALID_ARG;
+    if (batch > TOPK_STATIC_MAX_BATCH || (i64)batch * ceil_div(d, TK_CHUNK) > TOPK_STATIC_MAX_CHUNKS)
+        return EF21_ERR_UNSUPPORTED;                     // beyond the built-in scratch
+    TopkLayout L;
+    L.nchunks = (int)ceil_div(d, TK_CHUNK);
+    size_t o = 0;
+    L.state = o; o += align_up((size_t)batch * sizeof(TkState));
+    L.hist = o; o += align_up((size_t)batch * TK_BINS * sizeof(unsigned));
+    L.chunks = o; o += align_up((size_t)batch * (size_t)L.nchunks * sizeof(uint2));
+    L.fast = false; L.nreg = 0; L.thr = L.flags = L.slow_count = L.region_cnt = L.cand = 0;
+    L.total = o;
+    if (L.total > TOPK_STATIC_SCRATCH_BYTES) return EF21_ERR_UNSUPPORTED;
+    void* scratch = nullptr;
+    EF(topk_static_scratch(&scratch));
+    TopkBuffers B = topk_buffers(static_cast<char*>(scratch), L);
+    // tk_reset_kernel clears the selection state and the histograms of the vectors in use; the
+    // per-chunk counts are fully rewritten before they are read.
+    return enqueue_topk_general(reinterpret_cast<cudaStream_t>(cuda_stream), v_dev, d, nullptr, 0, batch, d, k,
+                                idx_out_dev, val_out_dev, B, nullptr);
 }
 
 static ef21_status copy_state_out(ef21_ctx* c, float* x, float* g, float* gi, int32_t* li, float* lv, cudaMemcpyKind kind) {
