@@ -1,7 +1,8 @@
 #!/usr/bin/env python
 """Benchmark of the EF21 hot path (libef21) on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--headline-only]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload all|headline|stress] [--stress-n N] [--no-cpu] [--no-e2e]
 
 A "step" is one EF21 iteration (Algorithm 2's loop body over all n workers).  The headline
 workload is the mushrooms-shaped logistic problem (n = 20, d = 112, N = 8,124, Top-1, gamma = 1/L);
@@ -64,28 +65,36 @@ class ClockSampler:
     def __init__(self, index: int):
         self.index = index
         self.rows = []
-        self._stop = threading.Event()
+        self.proc = None
         self._thread = threading.Thread(target=self._run, daemon=True)
 
     def _run(self):
-        while not self._stop.is_set():
-            try:
-                out = subprocess.run(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                                      "-i", str(self.index)], capture_output=True, text=True, timeout=5).stdout
-                parts = [p.strip() for p in out.strip().split(",")]
+        try:
+            for line in self.proc.stdout:
+                parts = [p.strip() for p in line.strip().split(",")]
                 if len(parts) >= 6:
                     self.rows.append(parts)
-            except Exception:
-                pass
-            self._stop.wait(0.05)
+        except Exception:
+            pass
 
     def __enter__(self):
-        self._thread.start()
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", "20"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self._thread.start()
+        except Exception:
+            self.proc = None
         return self
 
     def __exit__(self, *exc):
-        self._stop.set()
-        self._thread.join(timeout=10)
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+            self._thread.join(timeout=5)
 
     def summary(self):
         if not self.rows:
@@ -177,6 +186,46 @@ def run_ours(args):
 
     dev = lambda a: torch.as_tensor(np.ascontiguousarray(a)).to(device)
 
+    def time_stress(n_workers, steps, warmup):
+        ws = inputs.config(4)
+        n_w = n_workers or ws.n
+        V = torch.empty((n_w, ws.d), dtype=torch.float32, device=device)
+        for i in range(n_w):
+            V[i].copy_(torch.from_numpy(ws.worker_vector(i)))
+        hs = B.EF21(n_w, ws.d, ws.k, ws.gamma, device=device)
+        hs.init_grads(None, B.INIT_ZERO)
+        hs.step_grads(V, max(1, warmup))
+        hs.init_grads(None, B.INIT_ZERO)
+        hs.set_x(torch.zeros(ws.d, dtype=torch.float32, device=device))
+        flush_l2()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        l0 = hs.launch_count
+        e0.record(); hs.step_grads(V, steps); e1.record()
+        barrier()
+        ms = max_over_ranks(e0.elapsed_time(e1))
+        b = stress_bytes_per_iteration(n_w, ws.d, ws.k)
+        gbs = b * steps / (ms * 1e-3) / 1e9
+        return {"workload": f"configs[4] {ws.name}: n={n_w} d={ws.d} Top-{ws.k} supplied gradients (static)",
+                "iterations_per_s": steps / (ms * 1e-3), "us_per_iteration": ms / steps * 1e3, "steps": steps,
+                "algorithmic_bytes_per_iteration": b, "algorithmic_GBps": gbs, "frac_of_hbm_peak": gbs / peak,
+                "launches": hs.launch_count - l0, "fallbacks": hs.fallback_count(), "device_status": hs.poll()}
+
+    if args.workload == "stress":
+        r = time_stress(args.stress_n, args.steps if args.steps is not None else 50,
+                        args.warmup if args.warmup is not None else 3)
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": world * r["iterations_per_s"], "unit": UNIT, "n_gpus": world,
+                              "steps": r["steps"], "ms_per_step": r["us_per_iteration"] / 1e3, "dtype": "f32",
+                              "data": "synthetic", "config": {"workload": r["workload"]},
+                              "roofline": {"bound": "hbm", "achieved": r["algorithmic_GBps"], "peak": peak, "unit": "GB/s",
+                                           "frac": r["frac_of_hbm_peak"], "traffic": None, "peak_kind": f"of {peak_kind}",
+                                           "kernel": "st_collect_kernel (dominant) + sample/finish/aggregate"},
+                              "gpu_launches": r["launches"], "fallbacks": r["fallbacks"]}), flush=True)
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
     def time_logistic(w, k, steps, warmup, repeats=3, with_clocks=False):
         h = B.EF21(w.n, w.d, k, w.gamma, w.lam, total_rows=w.N, device=device)
         h.load_shards(dev(w.A), dev(w.y), w.row_offsets)
@@ -226,7 +275,8 @@ def run_ours(args):
     A_pin = torch.from_numpy(w.A).pin_memory()
     y_pin = torch.from_numpy(w.y).pin_memory()
     e2e_times = []
-    for rep in range(3):
+    xh = gh = np.zeros(w.d, dtype=np.float32)
+    for rep in range(0 if args.no_e2e else 3):
         flush_l2()
         barrier()
         t0 = time.perf_counter()
@@ -236,8 +286,8 @@ def run_ours(args):
         h2.step(steps)
         xh, gh, _, _, _ = h2.get_state_host(want_gi=False, messages=False)      # synchronises
         e2e_times.append(max_over_ranks((time.perf_counter() - t0) * 1e3))
-    e2e_ms = statistics.median(e2e_times)
-    e2e = {"value": world * steps / (e2e_ms * 1e-3), "unit": UNIT,
+    e2e_ms = statistics.median(e2e_times) if e2e_times else float("nan")
+    e2e = None if args.no_e2e else {"value": world * steps / (e2e_ms * 1e-3), "unit": UNIT,
            "h2d_bytes_per_step": (w.A.nbytes + w.y.nbytes) / steps, "d2h_bytes_per_step": (xh.nbytes + gh.nbytes) / steps,
            "note": f"create + load_shards_host + init + {steps} iterations + get_state_host, pinned host buffers; "
                    "bytes are per run divided by the iterations of the run"}
@@ -265,7 +315,7 @@ def run_ours(args):
         line["cpu_baseline"] = None
 
     # ---- the other named workloads (context; not the headline) -------------------------------
-    if not args.headline_only and world == 1:
+    if args.workload == "all" and world == 1:
         others = []
         for cfg, k in ((2, 1), (2, 4), (2, 16), (3, 1)):
             wk = inputs.config(cfg, k=k)
@@ -275,28 +325,7 @@ def run_ours(args):
             others.append({"workload": f"configs[{cfg}] {wk.name} Top-{k}", "iterations_per_s": wk.T / (rr["ms"] * 1e-3),
                            "us_per_iteration": rr["ms"] / wk.T * 1e3, "algorithmic_GBps": gbs, "frac_of_hbm_peak": gbs / peak,
                            "launches": rr["launches"], "persistent_shape": rr["shape"], "f_end": rr["f_end"]})
-        ws = inputs.config(4)
-        V = torch.empty((ws.n, ws.d), dtype=torch.float32, device=device)
-        for i in range(ws.n):
-            V[i].copy_(torch.from_numpy(ws.worker_vector(i)))
-        hs = B.EF21(ws.n, ws.d, ws.k, ws.gamma, device=device)
-        hs.init_grads(None, B.INIT_ZERO)
-        hs.step_grads(V, 3)
-        hs.init_grads(None, B.INIT_ZERO)
-        hs.set_x(torch.zeros(ws.d, dtype=torch.float32, device=device))
-        flush_l2()
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        l0 = hs.launch_count
-        e0.record(); hs.step_grads(V, ws.T); e1.record()
-        torch.cuda.synchronize()
-        ms = e0.elapsed_time(e1)
-        b = stress_bytes_per_iteration(ws.n, ws.d, ws.k)
-        gbs = b * ws.T / (ms * 1e-3) / 1e9
-        others.append({"workload": f"configs[4] {ws.name}: n={ws.n} d={ws.d} Top-{ws.k} supplied gradients",
-                       "iterations_per_s": ws.T / (ms * 1e-3), "us_per_iteration": ms / ws.T * 1e3,
-                       "algorithmic_GBps": gbs, "frac_of_hbm_peak": gbs / peak, "launches": hs.launch_count - l0,
-                       "device_status": hs.poll()})
+        others.append(time_stress(None, 50, 3))
         line["workloads"] = others
 
     if world > 1:
@@ -311,7 +340,11 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--headline-only", action="store_true", help="skip the other named workloads")
+    ap.add_argument("--workload", default="all", choices=["all", "headline", "stress"],
+                    help="all: headline line with the other workloads attached; headline: only the headline; "
+                         "stress: only the supplied-gradient workload (its own line; for profiling)")
+    ap.add_argument("--stress-n", type=int, default=None, help="workers of the stress workload (default 64)")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end timing")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle timing")
     args = ap.parse_args()
     if args.impl == "reference":
