@@ -81,6 +81,7 @@ aggregate_kernel(const int* __restrict__ idx, const float* __restrict__ val, con
 // Needs n <= AGG_STAGE_MAX_N; a tile with more than AGG_STAGE_CAP entries takes the direct loop.
 constexpr int AGG_STAGE_MAX_N = 1024;
 constexpr int AGG_STAGE_CAP = 3072;
+constexpr int AGG_OWNER_SCAN_MAX = 512;   // tiles with at most this many entries skip the per-worker loop
 
 template <bool UPDATE_X>
 __global__ void __launch_bounds__(AGG_BLOCK)
@@ -88,15 +89,18 @@ aggregate_staged_kernel(const int* __restrict__ idx, const float* __restrict__ v
                         int n, int k, int ntiles, i64 d, float inv_n, float gamma,
                         float* __restrict__ g, float* __restrict__ x) {
     __shared__ float s[AGG_TILE];
-    __shared__ unsigned char touched[AGG_TILE];
+    __shared__ __align__(4) unsigned short touched[AGG_TILE];   // staged entries per coordinate
     __shared__ int w_start[AGG_STAGE_MAX_N + 1];
     __shared__ int w_lo[AGG_STAGE_MAX_N];
     __shared__ unsigned short e_idx[AGG_STAGE_CAP];
     __shared__ float e_val[AGG_STAGE_CAP];
     __shared__ unsigned scratch[33];
+    __shared__ unsigned short multi[AGG_OWNER_SCAN_MAX];
+    __shared__ unsigned n_multi;
     const int b = blockIdx.x;
     const i64 j0 = (i64)b * AGG_TILE;
     for (int t = threadIdx.x; t < AGG_TILE; t += AGG_BLOCK) { s[t] = 0.f; touched[t] = 0; }
+    if (threadIdx.x == 0) n_multi = 0u;
     unsigned base = 0u;
     for (int c0 = 0; c0 < n; c0 += AGG_BLOCK) {
         const int i = c0 + threadIdx.x;
@@ -122,6 +126,39 @@ aggregate_staged_kernel(const int* __restrict__ idx, const float* __restrict__ v
             e_val[e] = val[src];
         }
         __syncthreads();
+        if (total <= AGG_OWNER_SCAN_MAX) {
+            // Few entries: count the entries per coordinate (16-bit counters, two per word).
+            unsigned* cnt32 = reinterpret_cast<unsigned*>(touched);
+            for (int e = threadIdx.x; e < total; e += AGG_BLOCK) {
+                const int t = e_idx[e];
+                atomicAdd(&cnt32[t >> 1], (t & 1) ? 0x10000u : 1u);
+            }
+            __syncthreads();
+            // coordinates hit once: the entry is the sum; entries of coordinates hit several times go
+            // to a short list and are resolved by whole warps below, in staged (= worker) order
+            for (int e = threadIdx.x; e < total; e += AGG_BLOCK) {
+                const int t = e_idx[e];
+                if (touched[t] == 1) s[t] = __fadd_rn(0.f, e_val[e]);
+                else { const unsigned q = atomicAdd(&n_multi, 1u); multi[q] = (unsigned short)e; }
+            }
+            __syncthreads();
+            const int nm = (int)n_multi;                 // <= total <= AGG_OWNER_SCAN_MAX
+            const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+            for (int q = warp; q < nm; q += AGG_BLOCK / 32) {
+                const int e = multi[q];
+                const int t = e_idx[e];
+                float acc = 0.f; bool owner = true, seen = false;
+                for (int base2 = 0; base2 < total; base2 += 32) {
+                    const int p = base2 + lane;
+                    unsigned m = __ballot_sync(0xffffffffu, p < total && e_idx[p] == t);
+                    if (m && !seen) { owner = (base2 + __ffs(m) - 1) == e; seen = true; }
+                    if (!owner) break;                       // warp-uniform
+                    while (m) { const int bit = __ffs(m) - 1; acc = __fadd_rn(acc, e_val[base2 + bit]); m &= m - 1; }
+                }
+                if (owner && lane == 0) s[t] = acc;
+            }
+            __syncthreads();
+        } else
         for (int i = 0; i < n; ++i) {
             const int lo = w_start[i], hi = w_start[i + 1];
             if (lo == hi) continue;                  // uniform: read from shared memory
@@ -143,16 +180,24 @@ aggregate_staged_kernel(const int* __restrict__ idx, const float* __restrict__ v
             __syncthreads();
         }
     }
-    for (int t = threadIdx.x; t < AGG_TILE; t += AGG_BLOCK) {
+    // dense part of the tile: all loads first, then the updates
+    constexpr int PER = AGG_TILE / AGG_BLOCK;
+    float gv[PER], xv[PER];
+#pragma unroll
+    for (int u = 0; u < PER; ++u) {
+        const int t = u * AGG_BLOCK + threadIdx.x;
         const i64 j = j0 + t;
-        if (j >= d) break;
-        if (UPDATE_X) {
-            const float gj = g[j];
-            x[j] = fmaf(-gamma, gj, x[j]);
-            if (touched[t]) g[j] = __fadd_rn(gj, __fmul_rn(s[t], inv_n));
-        } else if (touched[t]) {
-            g[j] = __fadd_rn(g[j], __fmul_rn(s[t], inv_n));
-        }
+        gv[u] = 0.f; xv[u] = 0.f;
+        if (j < d && (UPDATE_X || touched[t])) gv[u] = g[j];
+        if (UPDATE_X && j < d) xv[u] = x[j];
+    }
+#pragma unroll
+    for (int u = 0; u < PER; ++u) {
+        const int t = u * AGG_BLOCK + threadIdx.x;
+        const i64 j = j0 + t;
+        if (j >= d) continue;
+        if (UPDATE_X) x[j] = fmaf(-gamma, gv[u], xv[u]);
+        if (touched[t]) g[j] = __fadd_rn(gv[u], __fmul_rn(s[t], inv_n));
     }
 }
 

@@ -132,6 +132,8 @@ struct ef21_ctx {
     int pk_used_cluster, pk_used_rb, pk_used_src;
     unsigned spin_limit;
     bool force_general_topk;
+    cudaStream_t aux_stream;            // created on first use: overlaps the next threshold estimate
+    cudaEvent_t ev_fork, ev_join;
     i64 launches;
     std::vector<i64> row_off;
     std::vector<RowTile> tiles;
@@ -184,19 +186,28 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 
 // Exact Top-k of v = a - b for long vectors in one pass over a and b (see stress.cuh).  If gi_rows
 // is given, g_i += c_i is applied by the same kernel that writes the messages.
+// Threshold estimate of the one-pass Top-k (first of its three kernels).
+ef21_status enqueue_topk_fast_sample(cudaStream_t st, const float* a, i64 pitch_a, const float* b, i64 pitch_b,
+                                     int batch, i64 d, int k, const TopkBuffers& B, i64* launches) {
+    const i64 target = std::max<i64>(2 * (i64)k, (i64)k + 2048);
+    i64 rank = ceil_div(target * (i64)(ST_SAMPLE_BLOCKS * ST_SAMPLE_LEN), d);
+    rank = std::min<i64>(std::max<i64>(rank, 32), ST_SAMPLE_BLOCKS * ST_SAMPLE_LEN / 2);
+    st_sample_kernel<<<batch, ST_THREADS, 0, st>>>(a, pitch_a, b, pitch_b, d, (unsigned)rank, B.thr, B.flags);
+    if (launches) *launches += 1;
+    CU(cudaGetLastError());
+    return EF21_OK;
+}
+
 ef21_status enqueue_topk_fast(cudaStream_t st, const float* a, i64 pitch_a, const float* b, i64 pitch_b,
                               int batch, i64 d, int k, int* idx_out, float* val_out, float* gi_rows, i64 ld,
-                              const TopkBuffers& B, i64* launches) {
+                              const TopkBuffers& B, i64* launches, bool sampled = false) {
     static bool smem_set = false;
     const size_t finish_smem = (size_t)ST_CAND_CAP * 8 + 2048 * 4;
     if (!smem_set) {
         CU(cudaFuncSetAttribute(st_finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)finish_smem));
         smem_set = true;
     }
-    const i64 target = std::max<i64>(2 * (i64)k, (i64)k + 2048);
-    i64 rank = ceil_div(target * (i64)(ST_SAMPLE_BLOCKS * ST_SAMPLE_LEN), d);
-    rank = std::min<i64>(std::max<i64>(rank, 32), ST_SAMPLE_BLOCKS * ST_SAMPLE_LEN / 2);
-    st_sample_kernel<<<batch, ST_THREADS, 0, st>>>(a, pitch_a, b, pitch_b, d, (unsigned)rank, B.thr, B.flags);
+    if (!sampled) EF(enqueue_topk_fast_sample(st, a, pitch_a, b, pitch_b, batch, d, k, B, launches));
     dim3 grid((unsigned)ceil_div(B.nreg, ST_COLLECT_WARPS), (unsigned)batch);
     const bool vec = aligned16(a) && pitch_a % 4 == 0 && (!b || (aligned16(b) && pitch_b % 4 == 0));
     if (vec)
@@ -207,7 +218,7 @@ ef21_status enqueue_topk_fast(cudaStream_t st, const float* a, i64 pitch_a, cons
                                                                          B.region_cnt, B.flags);
     st_finish_kernel<<<batch, ST_THREADS, finish_smem, st>>>(a, pitch_a, b, pitch_b, d, B.nreg, k, B.cand, B.region_cnt,
                                                              B.flags, idx_out, val_out, gi_rows, ld, B.slow_count);
-    if (launches) *launches += 3;
+    if (launches) *launches += 2;
     CU(cudaGetLastError());
     return EF21_OK;
 }
@@ -247,13 +258,13 @@ ef21_status enqueue_grads(ef21_ctx* c, bool with_loss) {
     return EF21_OK;
 }
 
-// One message round: c_i = C(a_i - g_i), g_i += c_i, g += (1/n) sum c_i (and, if update_x,
-// x <- x - gamma g_old fused into the aggregation).
-ef21_status enqueue_round(ef21_ctx* c, const float* a, i64 pitch_a, bool update_x) {
+// Selection half of a message round: c_i = C(a_i - g_i) and g_i += c_i.  sampled: the threshold
+// kernel of the one-pass Top-k has already run for these inputs.
+ef21_status enqueue_round_select(ef21_ctx* c, const float* a, i64 pitch_a, bool sampled) {
     TopkBuffers B = topk_buffers(c->ws + c->L.topk, c->L.tk);
     if (B.fast && !c->force_general_topk) {
         EF(enqueue_topk_fast(c->stream, a, pitch_a, c->gi(), c->L.ld, c->n, c->d, c->k, c->msg_idx(), c->msg_val(),
-                             c->gi(), c->L.ld, B, &c->launches));
+                             c->gi(), c->L.ld, B, &c->launches, sampled));
     } else {
         EF(enqueue_topk_general(c->stream, a, pitch_a, c->gi(), c->L.ld, c->n, c->d, c->k, c->msg_idx(),
                                 c->msg_val(), B, &c->launches));
@@ -262,6 +273,12 @@ ef21_status enqueue_round(ef21_ctx* c, const float* a, i64 pitch_a, bool update_
                                                                                     c->k, c->L.ld, c->gi());
         c->launches += 1;
     }
+    CU(cudaGetLastError());
+    return EF21_OK;
+}
+
+// Aggregation half: g += (1/n) sum c_i (and, if update_x, x <- x - gamma g_old in the same kernel).
+ef21_status enqueue_round_aggregate(ef21_ctx* c, bool update_x) {
     const i64 noff = (i64)c->n * (c->L.agg_tiles + 1);
     agg_offsets_kernel<<<(unsigned)ceil_div(noff, 256), 256, 0, c->stream>>>(c->msg_idx(), c->n, c->k,
                                                                             c->L.agg_tiles, c->at<int>(c->L.agg_off));
@@ -274,6 +291,11 @@ ef21_status enqueue_round(ef21_ctx* c, const float* a, i64 pitch_a, bool update_
     c->launches += 2;
     CU(cudaGetLastError());
     return EF21_OK;
+}
+
+ef21_status enqueue_round(ef21_ctx* c, const float* a, i64 pitch_a, bool update_x) {
+    EF(enqueue_round_select(c, a, pitch_a, false));
+    return enqueue_round_aggregate(c, update_x);
 }
 
 ef21_status enqueue_x_update(ef21_ctx* c) {
@@ -511,6 +533,7 @@ ef21_status ef21_create(ef21_ctx** out, int32_t n, int64_t d, int32_t k, float g
     c->pk_used_cluster = c->pk_used_rb = 0; c->pk_used_src = -1;
     c->spin_limit = 1u << 22;
     c->force_general_topk = false;
+    c->aux_stream = nullptr; c->ev_fork = nullptr; c->ev_join = nullptr;
     cudaError_t e = cudaMemsetAsync(c->ws + L.status, 0, 256, c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->x(), 0, (size_t)L.ld * 4, c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->g(), 0, (size_t)L.ld * 4, c->stream);
@@ -523,7 +546,13 @@ ef21_status ef21_create(ef21_ctx** out, int32_t n, int64_t d, int32_t k, float g
     return EF21_OK;
 }
 
-void ef21_destroy(ef21_ctx* ctx) { delete ctx; }
+void ef21_destroy(ef21_ctx* ctx) {
+    if (!ctx) return;
+    if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+    if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
+    if (ctx->aux_stream) cudaStreamDestroy(ctx->aux_stream);
+    delete ctx;
+}
 
 ef21_status ef21_load_shards(ef21_ctx* c, const float* A_dev, const float* y_dev, const int64_t* row_offsets_host) {
     if (!c || !row_offsets_host) return EF21_ERR_INVALID_ARG;
@@ -598,7 +627,32 @@ ef21_status ef21_step(ef21_ctx* c, int32_t steps) {
 ef21_status ef21_step_grads(ef21_ctx* c, const float* V_dev, int32_t steps) {
     if (!c || !V_dev || steps < 0) return EF21_ERR_INVALID_ARG;
     if (!c->inited) return EF21_ERR_STATE;
-    for (int t = 0; t < steps; ++t) EF(enqueue_round(c, V_dev, c->d, true));
+    const bool fast = c->L.tk.fast && !c->force_general_topk;
+    if (fast && steps > 1 && !c->aux_stream) {
+        // V is the same at every step, so the threshold estimate of step t+1 only waits for the
+        // g_i update of step t and can run beside the aggregation of step t on a second stream.
+        if (cudaStreamCreateWithFlags(&c->aux_stream, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+            cudaGetLastError();
+            return EF21_ERR_CUDA;
+        }
+    }
+    TopkBuffers B = topk_buffers(c->ws + c->L.topk, c->L.tk);
+    bool sampled = false;
+    for (int t = 0; t < steps; ++t) {
+        EF(enqueue_round_select(c, V_dev, c->d, sampled));
+        sampled = false;
+        if (fast && t + 1 < steps) {
+            CU(cudaEventRecord(c->ev_fork, c->stream));
+            CU(cudaStreamWaitEvent(c->aux_stream, c->ev_fork, 0));
+            EF(enqueue_topk_fast_sample(c->aux_stream, V_dev, c->d, c->gi(), c->L.ld, c->n, c->d, c->k, B, &c->launches));
+            CU(cudaEventRecord(c->ev_join, c->aux_stream));
+            sampled = true;
+        }
+        EF(enqueue_round_aggregate(c, true));
+        if (sampled) CU(cudaStreamWaitEvent(c->stream, c->ev_join, 0));
+    }
     c->last_path = EF21_PATH_LAUNCHES;
     return EF21_OK;
 }

@@ -234,7 +234,8 @@ st_finish_kernel(const float* a, i64 pitch_a, const float* b, i64 pitch_b, i64 d
     float* __restrict__ vo = val_out + (i64)i * k;
     float* gi_row = gi_rows ? gi_rows + (i64)i * ld : nullptr;
 
-    // stage the candidates in index order
+    // stage the candidates in index order: per group of 1024 regions, prefix-sum the region counts,
+    // then copy with one thread per candidate (its region found by binary search in the prefix)
     unsigned total = 0u;
     bool bad = flags[i] != 0u;
     for (int r0 = 0; r0 < nreg; r0 += ST_THREADS) {
@@ -242,14 +243,34 @@ st_finish_kernel(const float* a, i64 pitch_a, const float* b, i64 pitch_b, i64 d
         const unsigned c = r < nreg ? (unsigned)region_cnt[(i64)i * nreg + r] : 0u;
         unsigned tot;
         const unsigned pre = block_excl_scan(c, scratch, tot);
-        if (!bad && c <= (unsigned)ST_REGION_CAP) {
-            const int2* __restrict__ src = cand + ((i64)i * nreg + r) * ST_REGION_CAP;
-            for (unsigned e = 0; e < c; ++e) {
-                const unsigned pos = total + pre + e;
-                if (pos < (unsigned)ST_CAND_CAP) { const int2 w = src[e]; cidx[pos] = w.x; cval[pos] = __int_as_float(w.y); }
+        hist[threadIdx.x] = pre;                      // hist doubles as the prefix array here
+        if (threadIdx.x == 0) hist[ST_THREADS] = tot;
+        __syncthreads();
+        if (!bad && total + tot <= (unsigned)ST_CAND_CAP) {
+            constexpr int U = 8;                         // candidates in flight per thread
+            for (unsigned eb = 0; eb < tot; eb += U * ST_THREADS) {
+                int2 w[U];
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const unsigned e = eb + u * ST_THREADS + threadIdx.x;
+                    if (e < tot) {
+                        int lo = 0, hi = ST_THREADS;     // last region with prefix <= e
+                        while (hi - lo > 1) {
+                            const int mid = (lo + hi) >> 1;
+                            if (hist[mid] <= e) lo = mid; else hi = mid;
+                        }
+                        w[u] = cand[((i64)i * nreg + r0 + lo) * ST_REGION_CAP + (e - hist[lo])];
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const unsigned e = eb + u * ST_THREADS + threadIdx.x;
+                    if (e < tot) { cidx[total + e] = w[u].x; cval[total + e] = __int_as_float(w[u].y); }
+                }
             }
         }
         total += tot;
+        __syncthreads();
     }
     __syncthreads();
     if (bad || total < (unsigned)k || total > (unsigned)ST_CAND_CAP) {
@@ -271,29 +292,48 @@ st_finish_kernel(const float* a, i64 pitch_a, const float* b, i64 pitch_b, i64 d
         select_advance(s, level, res);
         __syncthreads();
     }
-    unsigned ge_before = 0u, tie_before = 0u;
-    for (unsigned base = 0; base < total; base += ST_THREADS) {
-        const unsigned e = base + threadIdx.x;
-        float val = 0.f; int j = 0; unsigned is_ge = 0u, is_tie = 0u;
-        if (e < total) {
-            val = cval[e]; j = cidx[e];
-            const unsigned key = mag_key(val);
-            is_ge = key >= s.lo_ge ? 1u : 0u;
-            is_tie = (s.need_ties && key == s.T) ? 1u : 0u;
-        }
-        unsigned tot;
-        const unsigned packed = block_excl_scan(is_ge | (is_tie << 16), scratch, tot);
-        const unsigned my_ge = ge_before + (packed & 0xffffu), my_tie = tie_before + (packed >> 16);
-        const bool sel = is_ge || (is_tie && my_tie < s.need_ties);
-        if (sel) {
+    // ordered compaction: thread t owns the contiguous candidates [t*q, (t+1)*q)
+    const unsigned q = (total + ST_THREADS - 1) / ST_THREADS;
+    const unsigned e0 = min(threadIdx.x * q, total), e1 = min(e0 + q, total);
+    unsigned n_ge = 0u, n_tie = 0u;
+    for (unsigned e = e0; e < e1; ++e) {
+        const unsigned key = mag_key(cval[e]);
+        n_ge += key >= s.lo_ge ? 1u : 0u;
+        n_tie += (s.need_ties && key == s.T) ? 1u : 0u;
+    }
+    unsigned tot;
+    const unsigned packed = block_excl_scan(n_ge | (n_tie << 16), scratch, tot);
+    unsigned my_ge = packed & 0xffffu, my_tie = packed >> 16;
+    for (unsigned e = e0; e < e1; ++e) {
+        const float val = cval[e];
+        const unsigned key = mag_key(val);
+        const bool is_ge = key >= s.lo_ge;
+        const bool is_tie = s.need_ties && key == s.T;
+        if (is_ge || (is_tie && my_tie < s.need_ties)) {
             const unsigned pos = is_ge ? my_ge + min(my_tie, s.need_ties) : my_ge + my_tie;
-            if (pos < (unsigned)k) {
-                io[pos] = j; vo[pos] = val;
-                if (gi_row) gi_row[j] = __fadd_rn(gi_row[j], val);
-            }
+            if (pos < (unsigned)k) { io[pos] = cidx[e]; vo[pos] = val; }
         }
-        ge_before += tot & 0xffffu;
-        tie_before += tot >> 16;
+        my_ge += is_ge ? 1u : 0u;
+        my_tie += is_tie ? 1u : 0u;
+    }
+    if (gi_row) {
+        // g_i += c_i on the k selected coordinates (distinct), several read-modify-writes in flight
+        __syncthreads();
+        constexpr int U = 4;
+        for (int p0 = 0; p0 < k; p0 += U * ST_THREADS) {
+            int j[U]; float c[U], old[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int pp = p0 + u * ST_THREADS + threadIdx.x;
+                if (pp < k) { j[u] = io[pp]; c[u] = vo[pp]; }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+                if (p0 + u * ST_THREADS + (int)threadIdx.x < k) old[u] = gi_row[j[u]];
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+                if (p0 + u * ST_THREADS + (int)threadIdx.x < k) gi_row[j[u]] = __fadd_rn(old[u], c[u]);
+        }
     }
 }
 
