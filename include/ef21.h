@@ -176,7 +176,7 @@ ef21_status ef21_eval(ef21_ctx* ctx, double* f, double* grad_norm2, double* G);
 ef21_status ef21_poll(ef21_ctx* ctx);
 
 /* Top-k algorithm used inside the EF21 rounds of the launch path: 0 = automatic (long vectors,
- * d >= 2^18 and k <= 8192, take the one-pass path: sampled threshold, single streaming pass,
+ * d >= 2^18 and k <= 6144, take the one-pass path: sampled threshold, single streaming pass,
  * exact selection among the candidates; everything else takes the multi-pass radix select),
  * 1 = always the multi-pass radix select.  Both give the same bits. */
 ef21_status ef21_set_topk_algorithm(ef21_ctx* ctx, int32_t algorithm);

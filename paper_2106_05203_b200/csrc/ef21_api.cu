@@ -33,7 +33,7 @@ struct TopkLayout {
     // one-pass path for long vectors (stress.cuh); fast == false: sections absent
     bool fast;
     int nreg;
-    size_t thr, flags, slow_count, region_cnt, cand;
+    size_t thr, flags, done, slow_count, region_cnt, cand;
 };
 
 bool fast_topk_eligible(i64 d, i64 k) { return d >= ST_MIN_D && k <= ST_MAX_K; }
@@ -47,13 +47,14 @@ TopkLayout topk_layout(i64 batch, i64 d, i64 k) {
     L.chunks = o; o += align_up((size_t)batch * (size_t)L.nchunks * sizeof(uint2));
     L.fast = fast_topk_eligible(d, k);
     L.nreg = (int)ceil_div(d, ST_SUB);
-    L.thr = L.flags = L.slow_count = L.region_cnt = L.cand = 0;
+    L.thr = L.flags = L.done = L.slow_count = L.region_cnt = L.cand = 0;
     if (L.fast) {
         L.thr = o; o += align_up((size_t)batch * 4);
         L.flags = o; o += align_up((size_t)batch * 4);
+        L.done = o; o += align_up((size_t)batch * 4);
         L.slow_count = o; o += align_up(4);
         L.region_cnt = o; o += align_up((size_t)batch * L.nreg * 4);
-        L.cand = o; o += align_up((size_t)batch * L.nreg * ST_REGION_CAP * sizeof(int2));
+        L.cand = o; o += align_up((size_t)batch * L.nreg * ST_REGION_CAP * sizeof(int4));
     }
     L.total = o;
     return L;
@@ -164,7 +165,7 @@ namespace {
 struct TopkBuffers {
     TkState* state; unsigned* hist; uint2* chunks; int nchunks;
     bool fast; int nreg;
-    unsigned* thr; unsigned* flags; unsigned* slow_count; int* region_cnt; int2* cand;
+    unsigned* thr; unsigned* flags; unsigned* done; unsigned* slow_count; int* region_cnt; int4* cand;
 };
 
 TopkBuffers topk_buffers(char* base, const TopkLayout& L) {
@@ -176,16 +177,15 @@ TopkBuffers topk_buffers(char* base, const TopkLayout& L) {
     B.fast = L.fast; B.nreg = L.nreg;
     B.thr = reinterpret_cast<unsigned*>(base + L.thr);
     B.flags = reinterpret_cast<unsigned*>(base + L.flags);
+    B.done = reinterpret_cast<unsigned*>(base + L.done);
     B.slow_count = reinterpret_cast<unsigned*>(base + L.slow_count);
     B.region_cnt = reinterpret_cast<int*>(base + L.region_cnt);
-    B.cand = reinterpret_cast<int2*>(base + L.cand);
+    B.cand = reinterpret_cast<int4*>(base + L.cand);
     return B;
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-// Exact Top-k of v = a - b for long vectors in one pass over a and b (see stress.cuh).  If gi_rows
-// is given, g_i += c_i is applied by the same kernel that writes the messages.
 // Threshold estimate of the one-pass Top-k (first of its three kernels).
 ef21_status enqueue_topk_fast_sample(cudaStream_t st, const float* a, i64 pitch_a, const float* b, i64 pitch_b,
                                      int batch, i64 d, int k, const TopkBuffers& B, i64* launches) {
@@ -198,11 +198,13 @@ ef21_status enqueue_topk_fast_sample(cudaStream_t st, const float* a, i64 pitch_
     return EF21_OK;
 }
 
+// Exact Top-k of v = a - b for long vectors in one pass over a and b (see stress.cuh).  If gi_rows
+// is given, g_i += c_i is applied by the same kernel that writes the messages.
 ef21_status enqueue_topk_fast(cudaStream_t st, const float* a, i64 pitch_a, const float* b, i64 pitch_b,
                               int batch, i64 d, int k, int* idx_out, float* val_out, float* gi_rows, i64 ld,
                               const TopkBuffers& B, i64* launches, bool sampled = false) {
     static bool smem_set = false;
-    const size_t finish_smem = (size_t)ST_CAND_CAP * 8 + 2048 * 4;
+    const size_t finish_smem = (size_t)ST_CAND_CAP * 12 + 2048 * 4;
     if (!smem_set) {
         CU(cudaFuncSetAttribute(st_finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)finish_smem));
         smem_set = true;
@@ -210,12 +212,8 @@ ef21_status enqueue_topk_fast(cudaStream_t st, const float* a, i64 pitch_a, cons
     if (!sampled) EF(enqueue_topk_fast_sample(st, a, pitch_a, b, pitch_b, batch, d, k, B, launches));
     dim3 grid((unsigned)ceil_div(B.nreg, ST_COLLECT_WARPS), (unsigned)batch);
     const bool vec = aligned16(a) && pitch_a % 4 == 0 && (!b || (aligned16(b) && pitch_b % 4 == 0));
-    if (vec)
-        st_collect_kernel<true><<<grid, ST_COLLECT_WARPS * 32, 0, st>>>(a, pitch_a, b, pitch_b, d, B.nreg, B.thr, B.cand,
-                                                                        B.region_cnt, B.flags);
-    else
-        st_collect_kernel<false><<<grid, ST_COLLECT_WARPS * 32, 0, st>>>(a, pitch_a, b, pitch_b, d, B.nreg, B.thr, B.cand,
-                                                                         B.region_cnt, B.flags);
+    auto collect = vec ? st_collect_kernel<true> : st_collect_kernel<false>;
+    collect<<<grid, ST_COLLECT_WARPS * 32, 0, st>>>(a, pitch_a, b, pitch_b, d, B.nreg, B.thr, B.cand, B.region_cnt, B.flags);
     st_finish_kernel<<<batch, ST_THREADS, finish_smem, st>>>(a, pitch_a, b, pitch_b, d, B.nreg, k, B.cand, B.region_cnt,
                                                              B.flags, idx_out, val_out, gi_rows, ld, B.slow_count);
     if (launches) *launches += 2;

@@ -6,10 +6,12 @@
 //                the whole vector are expected to lie above.
 //   2. collect:  the single streaming pass.  Every warp owns a region of 4,096 consecutive entries
 //                and appends the entries with key >= tau_i to its own slot array, in index order
-//                (ballot ranks), so the candidate set of a vector is already sorted by index.
+//                (ballot ranks), so the candidate set of a vector is already sorted by index.  A
+//                record is (index, v, g_i + v): the updated state value travels with the candidate.
 //   3. finish:   one block per vector stages the candidates in shared memory, finds the exact k-th
 //                key by radix select, breaks ties toward the lower index by an ordered scan, writes
-//                the k pairs in ascending index order and applies g_i += c_i.
+//                the k pairs in ascending index order and stores g_i + c_i on the selected
+//                coordinates (no read-modify-write: the new value came with the candidate).
 // The threshold only decides speed, never the result: if a vector ends up with fewer than k
 // candidates, more than the staging capacity, or an overflowing region, its finish block runs the
 // exact selection over the whole vector instead (slow, same output bit for bit).
@@ -19,14 +21,20 @@
 namespace ef21 {
 
 constexpr int ST_SUB = 4096;            // entries per region (one warp)
-constexpr int ST_REGION_CAP = 256;      // candidate slots per region
+constexpr int ST_REGION_CAP = 128;      // candidate slots per region
 constexpr int ST_COLLECT_WARPS = 8;
+#ifndef ST_COLLECT_UNROLL
+#define ST_COLLECT_UNROLL 1
+#endif
+#ifndef ST_COLLECT_MIN_BLOCKS
+#define ST_COLLECT_MIN_BLOCKS 8
+#endif
 constexpr int ST_SAMPLE_BLOCKS = 64;
 constexpr int ST_SAMPLE_LEN = 1024;
 constexpr int ST_THREADS = 1024;        // sample / finish block size
-constexpr int ST_CAND_CAP = 24576;      // candidates staged in shared memory
+constexpr int ST_CAND_CAP = 16384;      // candidates staged in shared memory
 constexpr i64 ST_MIN_D = 262144;
-constexpr int ST_MAX_K = 8192;
+constexpr int ST_MAX_K = 6144;
 
 // All 1024 threads: given a 2048-bin histogram in shared memory (bins ordered by key digit), find
 // the bin that holds the need-th largest entry.  Returns bin, number of entries in higher bins,
@@ -82,76 +90,7 @@ st_sample_kernel(const float* __restrict__ a, i64 pitch_a, const float* __restri
 }
 
 // ---------------------------------------------------------------------------------------------
-// 2. the streaming pass
-// ---------------------------------------------------------------------------------------------
-template <bool VEC>
-__global__ void __launch_bounds__(ST_COLLECT_WARPS * 32)
-st_collect_kernel(const float* __restrict__ a, i64 pitch_a, const float* __restrict__ b, i64 pitch_b, i64 d,
-                  int nreg, const unsigned* __restrict__ thr, int2* __restrict__ cand,
-                  int* __restrict__ region_cnt, unsigned* __restrict__ flags) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int region = blockIdx.x * ST_COLLECT_WARPS + warp;
-    if (region >= nreg) return;
-    const int i = blockIdx.y;
-    const unsigned tau = thr[i];
-    const float* __restrict__ av = a + (i64)i * pitch_a;
-    const bool has_b = b != nullptr;
-    const float* __restrict__ bv = has_b ? b + (i64)i * pitch_b : av;
-    const i64 base = (i64)region * ST_SUB;
-    int2* __restrict__ out = cand + ((i64)i * nreg + region) * ST_REGION_CAP;
-    const unsigned lt = (1u << lane) - 1u;
-    int cnt = 0;
-    constexpr int UNROLL = 4;
-    for (int it0 = 0; it0 < ST_SUB / 128; it0 += UNROLL) {
-        float v[UNROLL][4];
-#pragma unroll
-        for (int u = 0; u < UNROLL; ++u) {
-            const i64 j0 = base + (i64)(it0 + u) * 128 + 4 * lane;
-            if (VEC && j0 + 3 < d) {
-                const float4 x4 = __ldcs(reinterpret_cast<const float4*>(av + j0));
-                if (has_b) {
-                    const float4 g4 = __ldcs(reinterpret_cast<const float4*>(bv + j0));
-                    v[u][0] = __fsub_rn(x4.x, g4.x); v[u][1] = __fsub_rn(x4.y, g4.y);
-                    v[u][2] = __fsub_rn(x4.z, g4.z); v[u][3] = __fsub_rn(x4.w, g4.w);
-                } else {
-                    v[u][0] = x4.x; v[u][1] = x4.y; v[u][2] = x4.z; v[u][3] = x4.w;
-                }
-            } else {
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    v[u][e] = (j0 + e < d) ? (has_b ? __fsub_rn(av[j0 + e], bv[j0 + e]) : av[j0 + e]) : 0.f;
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < UNROLL; ++u) {
-            const i64 j0 = base + (i64)(it0 + u) * 128 + 4 * lane;
-            bool pr[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) pr[e] = mag_key(v[u][e]) >= tau;
-            const unsigned any = __ballot_sync(0xffffffffu, pr[0] | pr[1] | pr[2] | pr[3]);
-            if (any) {
-                unsigned bm[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) bm[e] = __ballot_sync(0xffffffffu, pr[e]);
-                int pos = cnt + __popc(bm[0] & lt) + __popc(bm[1] & lt) + __popc(bm[2] & lt) + __popc(bm[3] & lt);
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    if (pr[e]) {
-                        if (pos < ST_REGION_CAP) out[pos] = make_int2((int)(j0 + e), __float_as_int(v[u][e]));
-                        ++pos;
-                    }
-                cnt += __popc(bm[0]) + __popc(bm[1]) + __popc(bm[2]) + __popc(bm[3]);
-            }
-        }
-    }
-    if (lane == 0) {
-        region_cnt[(i64)i * nreg + region] = cnt;
-        if (cnt > ST_REGION_CAP) atomicOr(&flags[i], 1u);
-    }
-}
-
-// ---------------------------------------------------------------------------------------------
-// 3. exact selection among the candidates (or, rarely, over the whole vector)
+// helpers of the exact selection (radix-select bookkeeping, whole-vector fallback)
 // ---------------------------------------------------------------------------------------------
 
 // Radix-select bookkeeping shared by the fast and the slow variant: digits of 11/10/10 bits.
@@ -215,21 +154,106 @@ __device__ void st_slow_exact(const float* av, const float* bv, i64 d, int k,
     }
 }
 
-// gi_rows: if not null, g_i[idx] += val is applied for the selected pairs (row pitch ld).
-__global__ void __launch_bounds__(ST_THREADS)
-st_finish_kernel(const float* a, i64 pitch_a, const float* b, i64 pitch_b, i64 d,
-                 int nreg, int k, const int2* __restrict__ cand, const int* __restrict__ region_cnt,
+// ---------------------------------------------------------------------------------------------
+// 2. the streaming pass
+// ---------------------------------------------------------------------------------------------
+// grid = (ceil(nreg / 8), batch), block = 256 threads: one warp per region of 4,096 entries.
+template <bool VEC>
+__global__ void __launch_bounds__(ST_COLLECT_WARPS * 32, ST_COLLECT_MIN_BLOCKS)
+st_collect_kernel(const float* __restrict__ a, i64 pitch_a, const float* __restrict__ b, i64 pitch_b, i64 d,
+                  int nreg, const unsigned* __restrict__ thr, int4* __restrict__ cand,
+                  int* __restrict__ region_cnt, unsigned* __restrict__ flags) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int i = blockIdx.y;
+    const float* __restrict__ av = a + (i64)i * pitch_a;
+    const bool has_b = b != nullptr;
+    const float* __restrict__ bv = has_b ? b + (i64)i * pitch_b : nullptr;
+    const int region = blockIdx.x * ST_COLLECT_WARPS + warp;
+    if (region < nreg) {
+        const unsigned tau = thr[i];
+        const i64 base = (i64)region * ST_SUB;
+        int4* out = cand + ((i64)i * nreg + region) * ST_REGION_CAP;
+        const unsigned lt = (1u << lane) - 1u;
+        int cnt = 0;
+        constexpr int UNROLL = ST_COLLECT_UNROLL;
+        for (int it0 = 0; it0 < ST_SUB / 128; it0 += UNROLL) {
+            float v[UNROLL][4], gold[UNROLL][4];
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const i64 j0 = base + (i64)(it0 + u) * 128 + 4 * lane;
+                if (VEC && j0 + 3 < d) {
+                    const float4 x4 = __ldcs(reinterpret_cast<const float4*>(av + j0));
+                    if (has_b) {
+                        const float4 g4 = __ldcs(reinterpret_cast<const float4*>(bv + j0));
+                        gold[u][0] = g4.x; gold[u][1] = g4.y; gold[u][2] = g4.z; gold[u][3] = g4.w;
+                        v[u][0] = __fsub_rn(x4.x, g4.x); v[u][1] = __fsub_rn(x4.y, g4.y);
+                        v[u][2] = __fsub_rn(x4.z, g4.z); v[u][3] = __fsub_rn(x4.w, g4.w);
+                    } else {
+                        gold[u][0] = gold[u][1] = gold[u][2] = gold[u][3] = 0.f;
+                        v[u][0] = x4.x; v[u][1] = x4.y; v[u][2] = x4.z; v[u][3] = x4.w;
+                    }
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        gold[u][e] = (has_b && j0 + e < d) ? bv[j0 + e] : 0.f;
+                        v[u][e] = (j0 + e < d) ? (has_b ? __fsub_rn(av[j0 + e], gold[u][e]) : av[j0 + e]) : 0.f;
+                    }
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const i64 j0 = base + (i64)(it0 + u) * 128 + 4 * lane;
+                bool pr[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) pr[e] = mag_key(v[u][e]) >= tau;
+                const unsigned any = __ballot_sync(0xffffffffu, pr[0] | pr[1] | pr[2] | pr[3]);
+                if (any) {
+                    unsigned bm[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) bm[e] = __ballot_sync(0xffffffffu, pr[e]);
+                    int pos = cnt + __popc(bm[0] & lt) + __popc(bm[1] & lt) + __popc(bm[2] & lt) + __popc(bm[3] & lt);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        if (pr[e]) {
+                            if (pos < ST_REGION_CAP) {
+                                const float gnew = __fadd_rn(gold[u][e], v[u][e]);
+                                out[pos] = make_int4((int)(j0 + e), __float_as_int(v[u][e]), __float_as_int(gnew), 0);
+                            }
+                            ++pos;
+                        }
+                    cnt += __popc(bm[0]) + __popc(bm[1]) + __popc(bm[2]) + __popc(bm[3]);
+                }
+            }
+        }
+        if (lane == 0) {
+            region_cnt[(i64)i * nreg + region] = cnt;
+            if (cnt > ST_REGION_CAP) atomicOr(&flags[i], 1u);
+        }
+    }
+
+}
+
+// ---------------------------------------------------------------------------------------------
+// 3. exact selection among the candidates (or, rarely, over the whole vector)
+// ---------------------------------------------------------------------------------------------
+// grid = batch, block = 1024 threads, dynamic shared memory = ST_CAND_CAP * 12 + 2048 * 4 bytes.
+// gi_rows: if not null, row i receives g_i + c_i on the selected coordinates (row pitch ld); b may
+// alias gi_rows.
+__global__ void __launch_bounds__(ST_THREADS, 1)
+st_finish_kernel(const float* a, i64 pitch_a, const float* b, i64 pitch_b, i64 d, int nreg, int k,
+                 const int4* __restrict__ cand, const int* __restrict__ region_cnt,
                  const unsigned* __restrict__ flags, int* __restrict__ idx_out, float* __restrict__ val_out,
                  float* gi_rows, i64 ld, unsigned* __restrict__ slow_count) {
     extern __shared__ __align__(16) unsigned char st_smem[];
-    int* cidx = reinterpret_cast<int*>(st_smem);                      // [ST_CAND_CAP]
-    float* cval = reinterpret_cast<float*>(cidx + ST_CAND_CAP);       // [ST_CAND_CAP]
-    unsigned* hist = reinterpret_cast<unsigned*>(cval + ST_CAND_CAP); // [2048]
     __shared__ unsigned scratch[33];
     __shared__ unsigned res[3];
     const int i = blockIdx.x;
     const float* av = a + (i64)i * pitch_a;
-    const float* bv = b ? b + (i64)i * pitch_b : nullptr;      // may alias gi_row
+    const float* bv = b ? b + (i64)i * pitch_b : nullptr;      // may alias the g_i row written below
+    int* cidx = reinterpret_cast<int*>(st_smem);                       // [ST_CAND_CAP]
+    float* cval = reinterpret_cast<float*>(cidx + ST_CAND_CAP);        // [ST_CAND_CAP]
+    float* cnew = cval + ST_CAND_CAP;                                  // [ST_CAND_CAP] g_i + v
+    unsigned* hist = reinterpret_cast<unsigned*>(cnew + ST_CAND_CAP);  // [2048]
     int* __restrict__ io = idx_out + (i64)i * k;
     float* __restrict__ vo = val_out + (i64)i * k;
     float* gi_row = gi_rows ? gi_rows + (i64)i * ld : nullptr;
@@ -244,12 +268,11 @@ st_finish_kernel(const float* a, i64 pitch_a, const float* b, i64 pitch_b, i64 d
         unsigned tot;
         const unsigned pre = block_excl_scan(c, scratch, tot);
         hist[threadIdx.x] = pre;                      // hist doubles as the prefix array here
-        if (threadIdx.x == 0) hist[ST_THREADS] = tot;
         __syncthreads();
         if (!bad && total + tot <= (unsigned)ST_CAND_CAP) {
             constexpr int U = 8;                         // candidates in flight per thread
             for (unsigned eb = 0; eb < tot; eb += U * ST_THREADS) {
-                int2 w[U];
+                int4 w[U];
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
                     const unsigned e = eb + u * ST_THREADS + threadIdx.x;
@@ -265,14 +288,16 @@ st_finish_kernel(const float* a, i64 pitch_a, const float* b, i64 pitch_b, i64 d
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
                     const unsigned e = eb + u * ST_THREADS + threadIdx.x;
-                    if (e < tot) { cidx[total + e] = w[u].x; cval[total + e] = __int_as_float(w[u].y); }
+                    if (e < tot) {
+                        cidx[total + e] = w[u].x; cval[total + e] = __int_as_float(w[u].y);
+                        cnew[total + e] = __int_as_float(w[u].z);
+                    }
                 }
             }
         }
         total += tot;
         __syncthreads();
     }
-    __syncthreads();
     if (bad || total < (unsigned)k || total > (unsigned)ST_CAND_CAP) {
         if (threadIdx.x == 0 && slow_count) atomicAdd(slow_count, 1u);
         st_slow_exact(av, bv, d, k, io, vo, gi_row, hist, scratch, res);
@@ -311,29 +336,14 @@ st_finish_kernel(const float* a, i64 pitch_a, const float* b, i64 pitch_b, i64 d
         const bool is_tie = s.need_ties && key == s.T;
         if (is_ge || (is_tie && my_tie < s.need_ties)) {
             const unsigned pos = is_ge ? my_ge + min(my_tie, s.need_ties) : my_ge + my_tie;
-            if (pos < (unsigned)k) { io[pos] = cidx[e]; vo[pos] = val; }
+            if (pos < (unsigned)k) {
+                const int j = cidx[e];
+                io[pos] = j; vo[pos] = val;
+                if (gi_row) gi_row[j] = cnew[e];           // g_i + c_i, computed when the entry was read
+            }
         }
         my_ge += is_ge ? 1u : 0u;
         my_tie += is_tie ? 1u : 0u;
-    }
-    if (gi_row) {
-        // g_i += c_i on the k selected coordinates (distinct), several read-modify-writes in flight
-        __syncthreads();
-        constexpr int U = 4;
-        for (int p0 = 0; p0 < k; p0 += U * ST_THREADS) {
-            int j[U]; float c[U], old[U];
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const int pp = p0 + u * ST_THREADS + threadIdx.x;
-                if (pp < k) { j[u] = io[pp]; c[u] = vo[pp]; }
-            }
-#pragma unroll
-            for (int u = 0; u < U; ++u)
-                if (p0 + u * ST_THREADS + (int)threadIdx.x < k) old[u] = gi_row[j[u]];
-#pragma unroll
-            for (int u = 0; u < U; ++u)
-                if (p0 + u * ST_THREADS + (int)threadIdx.x < k) gi_row[j[u]] = __fadd_rn(old[u], c[u]);
-        }
     }
 }
 

@@ -24,7 +24,8 @@ def _long_cases():
     cases = []
     cases.append(("student-262144-k1", inputs.stress_vector(5, 0, 262144), 1))
     cases.append(("student-262144-k262", inputs.stress_vector(5, 1, 262144), 262))
-    cases.append(("student-1m-k8192", inputs.stress_vector(5, 2, 1 << 20), 8192))
+    cases.append(("student-1m-k6144", inputs.stress_vector(5, 2, 1 << 20), 6144))
+    cases.append(("student-1m-k8192-multipass", inputs.stress_vector(5, 2, 1 << 20), 8192))
     cases.append(("gauss-unaligned-300001", rng.standard_normal(300001).astype(np.float32), 100))
     cases.append(("gauss-ragged-region-266245", rng.standard_normal(266245).astype(np.float32), 3000))
     v = (rng.integers(-4, 5, 400000)).astype(np.float32) * np.float32(0.25)        # nine magnitudes: huge tie classes
