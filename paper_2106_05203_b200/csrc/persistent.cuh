@@ -67,6 +67,37 @@ __device__ __forceinline__ unsigned ld_relaxed_u32(const unsigned* p) {
     return v;
 }
 
+// ---- distributed-shared-memory hand-off: remote stores that signal an mbarrier in the target block
+__device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ unsigned map_to_rank(unsigned addr, unsigned rank) {
+    unsigned r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void fence_mbar_init_cluster() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long* bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_parity(unsigned long long* bar, unsigned parity) {
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0u;
+}
+// 16-byte store into another block's shared memory; on arrival 16 bytes are credited to that block's mbarrier.
+__device__ __forceinline__ void st_async_f4(unsigned remote_dst, float4 v, unsigned remote_bar) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1, %2, %3, %4}, [%5];"
+                 ::"r"(remote_dst), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "r"(remote_bar) : "memory");
+}
+
 // Sum of v[r] over the 32 lanes for RB rows at once: after the call lane L holds the total of
 // row L / (32/RB).  RB-1 shuffles for the halving steps plus log2(32/RB) butterfly steps.
 template <int RB>
@@ -124,6 +155,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) persistent_kernel(const Persist
     unsigned long long* msg = reinterpret_cast<unsigned long long*>(part + C * ld);   // [nmsg]
     float* slice = reinterpret_cast<float*>(msg + ((nmsg + 1) & ~1));                  // SMEM source
     __shared__ int abort_flag;
+    __shared__ __align__(8) unsigned long long part_bar;     // leader: counts the bytes of the partials
 
     // ---- this block's rows --------------------------------------------------------------------
     const i64 w_r0 = p.row_off[worker], w_r1 = p.row_off[worker + 1];
@@ -133,7 +165,11 @@ __global__ void __launch_bounds__(PK_THREADS, 1) persistent_kernel(const Persist
     const int rows = (int)(r1 - r0);
     const int nbatch = (rows + RB - 1) / RB;
 
-    if (tid == 0) abort_flag = 0;
+    if (tid == 0) {
+        abort_flag = 0;
+        mbar_init(&part_bar, 1u);
+        fence_mbar_init_cluster();
+    }
     for (int j = tid; j < ld; j += PK_THREADS) { xs[j] = p.x[j]; gs[j] = p.g[j]; }
     if (SRC == PK_SRC_SMEM) {
         const float4* src = reinterpret_cast<const float4*>(p.A + r0 * (i64)ld);
@@ -169,7 +205,9 @@ __global__ void __launch_bounds__(PK_THREADS, 1) persistent_kernel(const Persist
         y_reg = myrow < rows ? __ldg(p.y + r0 + myrow) : 0.f;
     };
     if (SRC == PK_SRC_REG) load_batch(warp);     // host guarantees nbatch <= PK_WARPS
-    __syncthreads();
+    if (C > 1) cluster.sync(); else __syncthreads();        // barriers initialised before any remote store
+    const unsigned part_bytes = (unsigned)(C - 1) * (unsigned)chunks * 16u;
+    const unsigned remote_part = map_to_rank(smem_u32(part), 0u), remote_bar = map_to_rank(smem_u32(&part_bar), 0u);
 
     bool aborted = false;
     for (int t = 0; t < p.steps; ++t) {
@@ -178,12 +216,10 @@ __global__ void __launch_bounds__(PK_THREADS, 1) persistent_kernel(const Persist
 
         if (!aborted) {
             // 1. x <- x - gamma g on this block's replica (Algorithm 2, first line of the loop)
-            for (int j = tid; j < ld; j += PK_THREADS) {
-                const float xj = fmaf(-p.gamma, gs[j], xs[j]);
-                xs[j] = xj;
-                rterm[j] = regulariser_grad(p.lambda, xj);
-            }
+            for (int j = tid; j < ld; j += PK_THREADS) xs[j] = fmaf(-p.gamma, gs[j], xs[j]);
+            if (leader && C > 1 && tid == 0) mbar_arrive_expect_tx(&part_bar, part_bytes);
             __syncthreads();
+            for (int j = tid; j < ld; j += PK_THREADS) rterm[j] = regulariser_grad(p.lambda, xs[j]);
 
             // 2. partial gradient over this warp's batches
             float4 xr[CHUNKS], acc[CHUNKS];
@@ -219,16 +255,37 @@ __global__ void __launch_bounds__(PK_THREADS, 1) persistent_kernel(const Persist
             }
             __syncthreads();
 
-            // 3. block partial (warps in ascending order) -> leader's shared memory
-            float* leader_part = C > 1 ? cluster.map_shared_rank(part, 0) : part;
-            for (int j = tid; j < ld; j += PK_THREADS) {
-                float s = red[j];
+            // 3. block partial (warps in ascending order) -> leader's shared memory.  Remote blocks send
+            //    16-byte stores that credit the leader's barrier; they do not wait for anything.
+            for (int c = tid; c < chunks; c += PK_THREADS) {
+                float4 sum = reinterpret_cast<const float4*>(red)[c];
 #pragma unroll
-                for (int w = 1; w < PK_WARPS; ++w) s = __fadd_rn(s, red[w * ld + j]);
-                leader_part[crank * ld + j] = s;
+                for (int w = 1; w < PK_WARPS; ++w) {
+                    const float4 o = reinterpret_cast<const float4*>(red + w * ld)[c];
+                    sum.x = __fadd_rn(sum.x, o.x); sum.y = __fadd_rn(sum.y, o.y);
+                    sum.z = __fadd_rn(sum.z, o.z); sum.w = __fadd_rn(sum.w, o.w);
+                }
+                if (leader) reinterpret_cast<float4*>(part)[c] = sum;
+                else st_async_f4(remote_part + (unsigned)(crank * ld + 4 * c) * 4u, sum, remote_bar);
+            }
+            if (leader) {
+                __syncthreads();
+                if (C > 1) {
+                    // bounded: by tries and by elapsed clocks (about two seconds), whichever comes first
+                    unsigned spins = 0;
+                    const long long wait_t0 = clock64();
+                    while (!mbar_try_wait_parity(&part_bar, (unsigned)t & 1u)) {
+                        if (++spins > p.spin_limit || clock64() - wait_t0 > 4000000000ll) {
+                            record_error(p.status, 5u /* EF21_ERR_TIMEOUT */);
+                            abort_flag = 1;
+                            break;
+                        }
+                    }
+                    __syncthreads();
+                    if (abort_flag) aborted = true;
+                }
             }
         }
-        if (C > 1) cluster.sync(); else __syncthreads();
 
         if (!aborted) {
             // 4. leader: gradient, difference, Top-k, state update, publish
@@ -333,6 +390,10 @@ __global__ void __launch_bounds__(PK_THREADS, 1) persistent_kernel(const Persist
     }
 
     __syncthreads();
+    if (C > 1) {
+        if (aborted) __nanosleep(20000);         // let remote stores that were in flight land
+        cluster.sync();
+    }
     if (blockIdx.x == 0)
         for (int j = tid; j < ld; j += PK_THREADS) { p.x[j] = xs[j]; p.g[j] = gs[j]; }
     if (leader)
