@@ -391,7 +391,7 @@ struct PersistPlan {
 };
 
 size_t pk_smem_bytes(int ld, int C, int nmsg, int src, i64 rows_cta) {
-    size_t b = (size_t)(5 + PK_WARPS + C) * ld * 4 + (size_t)((nmsg + 1) & ~1) * 8;
+    size_t b = (size_t)(6 + PK_WARPS + C) * ld * 4 + (size_t)((nmsg + 1) & ~1) * 8 + (size_t)((2 * ld + 15) & ~15);
     if (src == PK_SRC_SMEM) b += (size_t)rows_cta * ld * 4;
     return b;
 }
@@ -411,8 +411,24 @@ PersistPlan plan_persistent(ef21_ctx* c) {
     i64 max_m = 0;
     for (int i = 0; i < c->n; ++i) max_m = std::max<i64>(max_m, c->row_off[i + 1] - c->row_off[i]);
     const int nmsg = c->n * c->k;
-    for (int C = 8; C >= 1; --C) {
-        if (c->pk_cluster > 0 && C != c->pk_cluster) continue;
+    // Order in which cluster sizes are tried: the smallest one that keeps a block's rows in registers with
+    // at most 16 rows per warp batch (fewer blocks = fewer senders and pollers), then the largest first.
+    int order[9], norder = 0;
+    if (c->pk_cluster > 0) {
+        order[norder++] = c->pk_cluster;
+    } else {
+        int pref = 0;
+        for (int C = 1; C <= 8 && !pref; ++C) {
+            if ((i64)c->n * C > sms) break;
+            const i64 rows = ceil_div(std::max<i64>(max_m, 1), C);
+            if (ceil_div(rows, std::min(16, max_rb)) <= PK_WARPS) pref = C;
+        }
+        if (pref) order[norder++] = pref;
+        for (int C = 8; C >= 1; --C)
+            if (C != pref) order[norder++] = C;
+    }
+    for (int oi = 0; oi < norder; ++oi) {
+        const int C = order[oi];
         if ((i64)c->n * C > sms) continue;
         const i64 rows_cta = ceil_div(std::max<i64>(max_m, 1), C);
         if (c->pk_cluster == 0 && C > 1 && rows_cta < 8) continue;       // do not split below one batch
@@ -420,7 +436,7 @@ PersistPlan plan_persistent(ef21_ctx* c) {
         for (int cand = 8; cand <= max_rb; cand *= 2)
             if (ceil_div(rows_cta, cand) <= PK_WARPS) { rb = cand; src = PK_SRC_REG; break; }
         if (rb == 0) {
-            rb = max_rb;
+            rb = std::min(max_rb, 16);
             src = pk_smem_bytes(ld, C, nmsg, PK_SRC_SMEM, rows_cta) <= (size_t)max_smem - 1024 ? PK_SRC_SMEM : PK_SRC_GMEM;
         }
         if (c->pk_rb > 0) {

@@ -10,13 +10,17 @@
 //   1. x <- fma(-gamma, g, x)                                   (every block, its replica)
 //   2. rows in batches of RB per warp: margins a_r.x by a transposed warp reduction (lane L ends
 //      up with the margin of row L/(32/RB)), residual rho_r, rank-1 accumulation rho_r a_r
-//   3. block partial -> leader block of the cluster through distributed shared memory
+//   3. block partial -> leader block of the cluster: 16-byte st.async stores into the leader's shared
+//      memory that credit an mbarrier there; the senders do not wait, the leader waits (bounded) for
+//      the byte count of all partials
 //   4. leader block: grad_i = sum/m_i + regulariser' and v = grad_i - g_i, one coordinate per
-//      thread; its warp 0 then takes Top-k by k rounds of a warp arg-max on (|v| bits, lower index
-//      wins), updates g_i += c_i and publishes k packed 64-bit words (epoch:16 | index:16 |
-//      value bits:32) into a double-buffered global slot array
-//   5. every block polls the n*k words of this iteration's epoch (bounded spin), then each
-//      coordinate thread adds the matching values in ascending worker order: g += (1/n) sum c_i
+//      thread; Top-k either by k rounds of a warp arg-max on (|v| bits, lower index wins) or, for
+//      larger k, by rank counting (every coordinate counts the entries ahead of it); g_i += c_i;
+//      k packed 64-bit words (epoch:16 | index:16 | value bits:32) go into a double-buffered global
+//      slot array
+//   5. every block polls the n*k words of this iteration's epoch (bounded spin); then each
+//      coordinate thread adds the matching values in ascending worker order (few messages), or warp 0
+//      folds the messages worker by worker into running sums (many messages): g += (1/n) sum c_i
 //
 // All summation orders are fixed by the launch shape, so two runs give identical bits.  A wait
 // that exceeds its spin limit records EF21_ERR_TIMEOUT in the status word; from then on every
@@ -33,6 +37,7 @@ constexpr int PK_THREADS = 256;
 constexpr int PK_WARPS = PK_THREADS / 32;
 constexpr int PK_MAX_K = 32;
 constexpr int PK_MAX_MSGS = 2048;       // n*k words staged in shared memory
+constexpr int PK_SCAN_MAX_MSGS = 128;   // up to this many messages every coordinate thread scans them all
 enum { PK_SRC_REG = 0, PK_SRC_SMEM = 1, PK_SRC_GMEM = 2 };
 
 struct PersistParams {
@@ -153,7 +158,10 @@ __global__ void __launch_bounds__(PK_THREADS, 1) persistent_kernel(const Persist
     float* red = vs + ld;                                           // [PK_WARPS][ld]
     float* part = red + PK_WARPS * ld;                              // [C][ld] (used in the leader)
     unsigned long long* msg = reinterpret_cast<unsigned long long*>(part + C * ld);   // [nmsg]
-    float* slice = reinterpret_cast<float*>(msg + ((nmsg + 1) & ~1));                  // SMEM source
+    float* sacc = reinterpret_cast<float*>(msg + ((nmsg + 1) & ~1));                  // [ld] per-coordinate sum of messages
+    unsigned char* touched = reinterpret_cast<unsigned char*>(sacc + ld);             // [ld] coordinate received a message
+    unsigned char* sel = touched + ld;                                                // [ld] leader: entry is in the Top-k
+    float* slice = reinterpret_cast<float*>(touched + ((2 * ld + 15) & ~15));         // SMEM source, 16-byte aligned
     __shared__ int abort_flag;
     __shared__ __align__(8) unsigned long long part_bar;     // leader: counts the bytes of the partials
 
@@ -171,6 +179,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) persistent_kernel(const Persist
         fence_mbar_init_cluster();
     }
     for (int j = tid; j < ld; j += PK_THREADS) { xs[j] = p.x[j]; gs[j] = p.g[j]; }
+    for (int j = tid; j < ld; j += PK_THREADS) { sacc[j] = 0.f; touched[j] = 0; }
     if (SRC == PK_SRC_SMEM) {
         const float4* src = reinterpret_cast<const float4*>(p.A + r0 * (i64)ld);
         float4* dst = reinterpret_cast<float4*>(slice);
@@ -209,6 +218,13 @@ __global__ void __launch_bounds__(PK_THREADS, 1) persistent_kernel(const Persist
     const unsigned part_bytes = (unsigned)(C - 1) * (unsigned)chunks * 16u;
     const unsigned remote_part = map_to_rank(smem_u32(part), 0u), remote_bar = map_to_rank(smem_u32(&part_bar), 0u);
 
+    const bool rank_select = p.k > 6;      // Top-k by rank counting instead of k arg-max rounds (cheaper from about 7 rounds on)
+    unsigned pad_mask = 0u;                // this lane's entries beyond d (chunk layout) can never be selected
+#pragma unroll
+    for (int cs = 0; cs < CHUNKS; ++cs)
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            if (4 * (lane + 32 * cs) + e >= p.d) pad_mask |= 1u << (cs * 4 + e);
     bool aborted = false;
     for (int t = 0; t < p.steps; ++t) {
         const unsigned epoch = (p.epoch0 + (unsigned)t + 1u) & 0xffffu;
@@ -219,7 +235,8 @@ __global__ void __launch_bounds__(PK_THREADS, 1) persistent_kernel(const Persist
             for (int j = tid; j < ld; j += PK_THREADS) xs[j] = fmaf(-p.gamma, gs[j], xs[j]);
             if (leader && C > 1 && tid == 0) mbar_arrive_expect_tx(&part_bar, part_bytes);
             __syncthreads();
-            for (int j = tid; j < ld; j += PK_THREADS) rterm[j] = regulariser_grad(p.lambda, xs[j]);
+            if (leader)
+                for (int j = tid; j < ld; j += PK_THREADS) rterm[j] = regulariser_grad(p.lambda, xs[j]);
 
             // 2. partial gradient over this warp's batches
             float4 xr[CHUNKS], acc[CHUNKS];
@@ -298,36 +315,77 @@ __global__ void __launch_bounds__(PK_THREADS, 1) persistent_kernel(const Persist
                     vs[j] = __fsub_rn(grad, gis[j]);
                 }
                 __syncthreads();
+                if (rank_select) {
+                    // larger k: every coordinate counts the entries that precede it in (|v| descending, index
+                    // ascending) order; the k entries of rank < k are the message
+                    for (int j = tid; j < ld; j += PK_THREADS) {
+                        unsigned char chosen = 0;
+                        if (j < p.d) {
+                            const unsigned kj = mag_key(vs[j]);
+                            int rank = 0;
+#pragma unroll 4
+                            for (int i = 0; i < p.d; ++i) {
+                                const unsigned ki = mag_key(vs[i]);
+                                rank += (ki > kj || (ki == kj && i < j)) ? 1 : 0;
+                            }
+                            chosen = rank < p.k ? 1 : 0;
+                        }
+                        sel[j] = chosen;
+                    }
+                    __syncthreads();
+                }
             }
-            if (leader && warp == 0) {
+            if (leader && warp == 0 && rank_select) {
+                // ascending index order falls out of the ballot ranks
+                int base = 0;
+                for (int j0 = 0; j0 < ld; j0 += 32) {
+                    const int j = j0 + lane;
+                    const bool chosen = j < ld && sel[j] != 0;
+                    const unsigned bal = __ballot_sync(0xffffffffu, chosen);
+                    if (chosen) {
+                        const int pos = base + __popc(bal & ((1u << lane) - 1u));
+                        const float val = vs[j];
+                        gis[j] = __fadd_rn(gis[j], val);
+                        const unsigned long long word = ((unsigned long long)epoch << 48) | ((unsigned long long)(unsigned)j << 32) |
+                                                        (unsigned long long)__float_as_uint(val);
+                        st_relaxed_u64(slot + worker * p.k + pos, word);
+                        if (t == p.steps - 1) { p.msg_idx[worker * p.k + pos] = j; p.msg_val[worker * p.k + pos] = val; }
+                    }
+                    base += __popc(bal);
+                }
+            }
+            if (leader && warp == 0 && !rank_select) {
                 float4 v[CHUNKS];
-                unsigned taken = 0u;                  // bit (cs*4+comp) set: not selectable
+                unsigned taken = pad_mask;            // bit (cs*4+comp) set: not selectable
 #pragma unroll
                 for (int cs = 0; cs < CHUNKS; ++cs) {
                     const int c = lane + 32 * cs;
                     v[cs] = c < chunks ? reinterpret_cast<const float4*>(vs)[c] : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-                    for (int e = 0; e < 4; ++e)
-                        if (4 * c + e >= p.d) taken |= 1u << (cs * 4 + e);
                 }
                 int my_idx = 0; float my_val = 0.f;          // lane t keeps the t-th pick
                 for (int t2 = 0; t2 < p.k; ++t2) {
-                    long long best = -1;
+                    // arg-max of (|v| bits, lower index first): warp maximum of the key, then warp minimum of
+                    // the index among the entries that hold it
+                    int lk = -1;
 #pragma unroll
                     for (int cs = 0; cs < CHUNKS; ++cs)
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            const unsigned idx = (unsigned)(4 * (lane + 32 * cs) + e);
-                            const long long comp = ((long long)mag_key(comp_of(v[cs], e)) << 32) | (long long)(0xffffffffu - idx);
                             const bool ok = !((taken >> (cs * 4 + e)) & 1u);
-                            best = (ok && comp > best) ? comp : best;
+                            const int key = (int)mag_key(comp_of(v[cs], e));
+                            lk = (ok && key > lk) ? key : lk;
                         }
+                    const int wk = __reduce_max_sync(0xffffffffu, lk);
+                    unsigned li = 0xffffffffu;
 #pragma unroll
-                    for (int off = 16; off >= 1; off >>= 1) {
-                        const long long o = __shfl_xor_sync(0xffffffffu, best, off);
-                        best = o > best ? o : best;
-                    }
-                    const unsigned widx = 0xffffffffu - (unsigned)(best & 0xffffffffll);
+                    for (int cs = 0; cs < CHUNKS; ++cs)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const bool ok = !((taken >> (cs * 4 + e)) & 1u);
+                            const unsigned idx = (unsigned)(4 * (lane + 32 * cs) + e);
+                            if (ok && (int)mag_key(comp_of(v[cs], e)) == wk) li = min(li, idx);
+                        }
+                    const unsigned widx = __reduce_min_sync(0xffffffffu, li);
                     const int wchunk = (int)(widx >> 2), wlane = wchunk & 31, wcs = wchunk >> 5, we = (int)(widx & 3u);
                     float wval = 0.f;
 #pragma unroll
@@ -342,7 +400,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) persistent_kernel(const Persist
                 }
                 // ascending index order inside the message
                 int rank = 0;
-                for (int u = 0; u < p.k; ++u) {
+                for (int u = 0; u < p.k && p.k > 1; ++u) {
                     const int oi = __shfl_sync(0xffffffffu, my_idx, u);
                     rank += (lane < p.k && oi < my_idx) ? 1 : 0;
                 }
@@ -374,7 +432,27 @@ __global__ void __launch_bounds__(PK_THREADS, 1) persistent_kernel(const Persist
             __syncthreads();
             if (abort_flag) aborted = true;
         }
-        if (!aborted) {
+        if (!aborted && nmsg > PK_SCAN_MAX_MSGS) {
+            // many messages: warp 0 folds them into per-coordinate running sums, one worker at a time (a
+            // worker's k <= 32 coordinates are distinct), then every coordinate applies its sum
+            if (warp == 0) {
+                const int kk = p.k;
+                for (int i = 0; i < p.n; ++i) {
+                    if (lane < kk) {
+                        const unsigned long long w = msg[i * kk + lane];
+                        const unsigned idx = (unsigned)(w >> 32) & 0xffffu;
+                        if (idx < (unsigned)ld) { sacc[idx] = __fadd_rn(sacc[idx], __uint_as_float((unsigned)w)); touched[idx] = 1; }
+                    }
+                    __syncwarp();
+                }
+            }
+            __syncthreads();
+            for (int j = tid; j < p.d; j += PK_THREADS)
+                if (touched[j]) {
+                    gs[j] = __fadd_rn(gs[j], __fmul_rn(sacc[j], p.inv_n));
+                    sacc[j] = 0.f; touched[j] = 0;
+                }
+        } else if (!aborted) {
             // g_j += (1/n) * sum over workers (ascending) of the values sent for coordinate j
             for (int j = tid; j < p.d; j += PK_THREADS) {
                 float s = 0.f; bool touched = false;
