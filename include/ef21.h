@@ -193,7 +193,7 @@ ef21_status ef21_clear_status(ef21_ctx* ctx);
 ef21_status ef21_selftest_bounded_wait(ef21_ctx* ctx, uint32_t spin_limit);
 
 /* Tuning of the persistent path (Algorithm 2 as one kernel; worker i = one thread-block
- * cluster): blocks per cluster (1..8, 0 = automatic), rows per warp batch (8, 16, 32, 0 =
+ * cluster): blocks per cluster (1..8, 0 = automatic), rows per warp batch (4, 8, 16, 32, 0 =
  * automatic) and where the shard rows live (0 registers, 1 shared memory, 2 global memory /
  * L2, -1 = automatic).  A shape that cannot run makes ef21_step fall back (path AUTO) or
  * return EF21_ERR_UNSUPPORTED (path PERSISTENT).  get_ reports what the last persistent
@@ -202,6 +202,11 @@ ef21_status ef21_set_persistent_shape(ef21_ctx* ctx, int32_t cluster_blocks, int
                                       int32_t row_source);
 ef21_status ef21_get_persistent_shape(const ef21_ctx* ctx, int32_t* cluster_blocks,
                                       int32_t* rows_per_batch, int32_t* row_source);
+
+/* Threads per block of the persistent path: 256, 512 or 0 = automatic (512 exists only for batches
+ * of at most 16 float4 registers per lane).  get_ reports what the last persistent launch used. */
+ef21_status ef21_set_persistent_threads(ef21_ctx* ctx, int32_t threads_per_block);
+int32_t ef21_get_persistent_threads(const ef21_ctx* ctx);
 
 /* Forces an execution path (EF21_PATH_*) for later ef21_step calls. */
 ef21_status ef21_set_path(ef21_ctx* ctx, int32_t path);

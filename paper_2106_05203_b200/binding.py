@@ -53,6 +53,8 @@ SIGNATURES = {
     "ef21_selftest_bounded_wait": (ctypes.c_int, [_vp, ctypes.c_uint32]),
     "ef21_set_persistent_shape": (ctypes.c_int, [_vp, _i32, _i32, _i32]),
     "ef21_get_persistent_shape": (ctypes.c_int, [_vp, ctypes.POINTER(_i32), ctypes.POINTER(_i32), ctypes.POINTER(_i32)]),
+    "ef21_set_persistent_threads": (ctypes.c_int, [_vp, _i32]),
+    "ef21_get_persistent_threads": (_i32, [_vp]),
     "ef21_set_path": (ctypes.c_int, [_vp, _i32]),
     "ef21_last_path": (_i32, [_vp]),
     "ef21_launch_count": (_i64, [_vp]),
@@ -251,6 +253,12 @@ class EF21:
         _check(_lib.ef21_get_persistent_shape(self._h, ctypes.byref(c), ctypes.byref(r), ctypes.byref(s)),
                "ef21_get_persistent_shape")
         return c.value, r.value, s.value
+
+    def set_persistent_threads(self, threads_per_block: int) -> None:
+        _check(_lib.ef21_set_persistent_threads(self._h, threads_per_block), "ef21_set_persistent_threads")
+
+    def get_persistent_threads(self) -> int:
+        return int(_lib.ef21_get_persistent_threads(self._h))
 
     def set_path(self, path: int) -> None:
         _check(_lib.ef21_set_path(self._h, path), "ef21_set_path")

@@ -129,8 +129,8 @@ struct ef21_ctx {
     bool shards_loaded, inited;
     int num_tiles;
     int path, last_path;
-    int pk_cluster, pk_rb, pk_src;      // forced persistent-kernel shape (0 / -1 = automatic)
-    int pk_used_cluster, pk_used_rb, pk_used_src;
+    int pk_cluster, pk_rb, pk_src, pk_threads;      // forced persistent-kernel shape (0 / -1 = automatic)
+    int pk_used_cluster, pk_used_rb, pk_used_src, pk_used_threads;
     unsigned spin_limit;
     bool force_general_topk;
     cudaStream_t aux_stream;            // created on first use: overlaps the next threshold estimate
@@ -363,40 +363,53 @@ ef21_status finish_load(ef21_ctx* c, const i64* row_offsets_host) {
 
 typedef void (*PersistKernel)(const PersistParams);
 
-template <int CHUNKS, int RB>
+template <int CHUNKS, int RB, int THREADS>
 PersistKernel pk_by_src(int src) {
-    if (src == PK_SRC_REG) return persistent_kernel<CHUNKS, RB, PK_SRC_REG>;
-    if (src == PK_SRC_SMEM) return persistent_kernel<CHUNKS, RB, PK_SRC_SMEM>;
-    return persistent_kernel<CHUNKS, RB, PK_SRC_GMEM>;
+    if (src == PK_SRC_REG) return persistent_kernel<CHUNKS, RB, PK_SRC_REG, THREADS>;
+    if (src == PK_SRC_SMEM) return persistent_kernel<CHUNKS, RB, PK_SRC_SMEM, THREADS>;
+    return persistent_kernel<CHUNKS, RB, PK_SRC_GMEM, THREADS>;
 }
 
-PersistKernel pk_lookup(int chunks, int rb, int src) {
-    switch (chunks * 100 + rb) {
-        case 108: return pk_by_src<1, 8>(src);
-        case 116: return pk_by_src<1, 16>(src);
-        case 132: return pk_by_src<1, 32>(src);
-        case 208: return pk_by_src<2, 8>(src);
-        case 216: return pk_by_src<2, 16>(src);
-        case 308: return pk_by_src<3, 8>(src);
-        case 408: return pk_by_src<4, 8>(src);
+// Instantiated shapes: (chunk slots per lane, rows per warp batch, threads per block).  512 threads
+// leave 128 registers per thread, so they exist only where a batch needs at most 16 float4 registers.
+PersistKernel pk_lookup(int chunks, int rb, int src, int threads) {
+    switch (chunks * 10000 + rb * 100 + threads / 256) {
+        case 10401: return pk_by_src<1, 4, 256>(src);
+        case 10801: return pk_by_src<1, 8, 256>(src);
+        case 11601: return pk_by_src<1, 16, 256>(src);
+        case 13201: return pk_by_src<1, 32, 256>(src);
+        case 20401: return pk_by_src<2, 4, 256>(src);
+        case 20801: return pk_by_src<2, 8, 256>(src);
+        case 21601: return pk_by_src<2, 16, 256>(src);
+        case 30401: return pk_by_src<3, 4, 256>(src);
+        case 30801: return pk_by_src<3, 8, 256>(src);
+        case 40401: return pk_by_src<4, 4, 256>(src);
+        case 40801: return pk_by_src<4, 8, 256>(src);
+        case 10402: return pk_by_src<1, 4, 512>(src);
+        case 10802: return pk_by_src<1, 8, 512>(src);
+        case 11602: return pk_by_src<1, 16, 512>(src);
+        case 20402: return pk_by_src<2, 4, 512>(src);
+        case 20802: return pk_by_src<2, 8, 512>(src);
+        case 30402: return pk_by_src<3, 4, 512>(src);
+        case 40402: return pk_by_src<4, 4, 512>(src);
     }
     return nullptr;
 }
 
 struct PersistPlan {
     bool ok;
-    int C, rb, src, chunks;
+    int C, rb, src, chunks, threads;
     size_t smem;
     PersistKernel kernel;
 };
 
-size_t pk_smem_bytes(int ld, int C, int nmsg, int src, i64 rows_cta) {
-    size_t b = (size_t)(6 + PK_WARPS + C) * ld * 4 + (size_t)((nmsg + 1) & ~1) * 8 + (size_t)((2 * ld + 15) & ~15);
+size_t pk_smem_bytes(int ld, int C, int nmsg, int src, i64 rows_cta, int threads) {
+    size_t b = (size_t)(6 + threads / 32 + C) * ld * 4 + (size_t)((nmsg + 1) & ~1) * 8 + (size_t)((2 * ld + 15) & ~15);
     if (src == PK_SRC_SMEM) b += (size_t)rows_cta * ld * 4;
     return b;
 }
 
-// Chooses cluster size, rows per batch and the source of the shard rows; checks that all n
+// Chooses cluster size, block size, rows per batch and the source of the shard rows; checks that all n
 // clusters can be resident at once (the blocks wait on one another through global memory).
 PersistPlan plan_persistent(ef21_ctx* c) {
     PersistPlan P; P.ok = false;
@@ -407,12 +420,41 @@ PersistPlan plan_persistent(ef21_ctx* c) {
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
     const int chunk_slots = (ld / 4 + 31) / 32;
-    const int max_rb = chunk_slots == 1 ? 32 : (chunk_slots == 2 ? 16 : 8);
+    const int max_rb256 = chunk_slots == 1 ? 32 : (chunk_slots == 2 ? 16 : 8);      // rb * chunk_slots <= 32
+    const int max_rb512 = chunk_slots == 1 ? 16 : (chunk_slots == 2 ? 8 : 4);       // rb * chunk_slots <= 16
     i64 max_m = 0;
     for (int i = 0; i < c->n; ++i) max_m = std::max<i64>(max_m, c->row_off[i + 1] - c->row_off[i]);
     const int nmsg = c->n * c->k;
-    // Order in which cluster sizes are tried: the smallest one that keeps a block's rows in registers with
-    // at most 16 rows per warp batch (fewer blocks = fewer senders and pollers), then the largest first.
+
+    // One candidate shape for a cluster size: rows in registers with 8 warps if they fit, else with 16
+    // warps, else staged in shared memory or streamed from L2 with 16 warps.
+    auto shape_for = [&](int C, int& rb, int& src, int& threads) {
+        const i64 rows_cta = ceil_div(std::max<i64>(max_m, 1), C);
+        rb = 0;
+        for (int cand = 8; cand <= max_rb256 && !rb; cand *= 2)
+            if (ceil_div(rows_cta, cand) <= 8) { rb = cand; src = PK_SRC_REG; threads = 256; }
+        for (int cand = 4; cand <= max_rb512 && !rb; cand *= 2)
+            if (ceil_div(rows_cta, cand) <= 16) { rb = cand; src = PK_SRC_REG; threads = 512; }
+        if (!rb) {
+            rb = max_rb512; threads = 512;
+            src = pk_smem_bytes(ld, C, nmsg, PK_SRC_SMEM, rows_cta, threads) <= (size_t)max_smem - 1024 ? PK_SRC_SMEM : PK_SRC_GMEM;
+        }
+        if (c->pk_threads > 0) {
+            threads = c->pk_threads;
+            const int cap = threads == 512 ? max_rb512 : max_rb256;
+            if (rb > cap) rb = cap;
+            if (src == PK_SRC_REG && ceil_div(rows_cta, rb) > threads / 32) src = PK_SRC_SMEM;
+        }
+        if (c->pk_rb > 0) {
+            rb = c->pk_rb;
+            if (src == PK_SRC_REG && ceil_div(rows_cta, rb) > threads / 32) src = PK_SRC_SMEM;
+        }
+        if (c->pk_src >= 0) src = c->pk_src;
+        return rows_cta;
+    };
+
+    // Order in which cluster sizes are tried: the smallest one that keeps a block's rows in registers
+    // (fewer blocks = fewer senders and pollers), then the largest first.
     int order[9], norder = 0;
     if (c->pk_cluster > 0) {
         order[norder++] = c->pk_cluster;
@@ -420,8 +462,9 @@ PersistPlan plan_persistent(ef21_ctx* c) {
         int pref = 0;
         for (int C = 1; C <= 8 && !pref; ++C) {
             if ((i64)c->n * C > sms) break;
-            const i64 rows = ceil_div(std::max<i64>(max_m, 1), C);
-            if (ceil_div(rows, std::min(16, max_rb)) <= PK_WARPS) pref = C;
+            int rb, src, threads;
+            shape_for(C, rb, src, threads);
+            if (src == PK_SRC_REG && threads == 256 && rb <= 16) pref = C;
         }
         if (pref) order[norder++] = pref;
         for (int C = 8; C >= 1; --C)
@@ -430,34 +473,20 @@ PersistPlan plan_persistent(ef21_ctx* c) {
     for (int oi = 0; oi < norder; ++oi) {
         const int C = order[oi];
         if ((i64)c->n * C > sms) continue;
-        const i64 rows_cta = ceil_div(std::max<i64>(max_m, 1), C);
+        int rb = 0, src = PK_SRC_GMEM, threads = 256;
+        const i64 rows_cta = shape_for(C, rb, src, threads);
         if (c->pk_cluster == 0 && C > 1 && rows_cta < 8) continue;       // do not split below one batch
-        int rb = 0, src = PK_SRC_GMEM;
-        for (int cand = 8; cand <= max_rb; cand *= 2)
-            if (ceil_div(rows_cta, cand) <= PK_WARPS) { rb = cand; src = PK_SRC_REG; break; }
-        if (rb == 0) {
-            rb = std::min(max_rb, 16);
-            src = pk_smem_bytes(ld, C, nmsg, PK_SRC_SMEM, rows_cta) <= (size_t)max_smem - 1024 ? PK_SRC_SMEM : PK_SRC_GMEM;
-        }
-        if (c->pk_rb > 0) {
-            if (c->pk_rb > max_rb) continue;
-            rb = c->pk_rb;
-            if (src == PK_SRC_REG && ceil_div(rows_cta, rb) > PK_WARPS) src = PK_SRC_SMEM;
-        }
-        if (c->pk_src >= 0) {
-            if (c->pk_src == PK_SRC_REG && ceil_div(rows_cta, rb) > PK_WARPS) continue;
-            src = c->pk_src;
-        }
-        const size_t smem = pk_smem_bytes(ld, C, nmsg, src, rows_cta);
+        if (src == PK_SRC_REG && ceil_div(rows_cta, rb) > threads / 32) continue;
+        const size_t smem = pk_smem_bytes(ld, C, nmsg, src, rows_cta, threads);
         if (smem > (size_t)max_smem - 1024) continue;
-        PersistKernel kern = pk_lookup(chunk_slots, rb, src);
+        PersistKernel kern = pk_lookup(chunk_slots, rb, src, threads);
         if (!kern) continue;
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
             cudaGetLastError();
             continue;
         }
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)(c->n * C)); cfg.blockDim = dim3(PK_THREADS); cfg.dynamicSmemBytes = smem;
+        cfg.gridDim = dim3((unsigned)(c->n * C)); cfg.blockDim = dim3((unsigned)threads); cfg.dynamicSmemBytes = smem;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = (unsigned)C; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
@@ -465,7 +494,7 @@ PersistPlan plan_persistent(ef21_ctx* c) {
         int active = 0;
         if (cudaOccupancyMaxActiveClusters(&active, kern, &cfg) != cudaSuccess) { cudaGetLastError(); continue; }
         if (active < c->n) continue;
-        P.ok = true; P.C = C; P.rb = rb; P.src = src; P.chunks = chunk_slots; P.smem = smem; P.kernel = kern;
+        P.ok = true; P.C = C; P.rb = rb; P.src = src; P.chunks = chunk_slots; P.threads = threads; P.smem = smem; P.kernel = kern;
         return P;
     }
     return P;
@@ -481,7 +510,7 @@ ef21_status run_persistent(ef21_ctx* c, const PersistPlan& P, int steps) {
     p.spin_limit = c->spin_limit; p.epoch0 = 0u;
     CU(cudaMemsetAsync(p.slots, 0, (size_t)2 * c->n * c->k * 8, c->stream));
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(c->n * P.C)); cfg.blockDim = dim3(PK_THREADS); cfg.dynamicSmemBytes = P.smem;
+    cfg.gridDim = dim3((unsigned)(c->n * P.C)); cfg.blockDim = dim3((unsigned)P.threads); cfg.dynamicSmemBytes = P.smem;
     cfg.stream = c->stream;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -497,7 +526,7 @@ ef21_status run_persistent(ef21_ctx* c, const PersistPlan& P, int steps) {
     }
     if (e != cudaSuccess) { cudaGetLastError(); return EF21_ERR_CUDA; }
     c->launches += 1;
-    c->pk_used_cluster = P.C; c->pk_used_rb = P.rb; c->pk_used_src = P.src;
+    c->pk_used_cluster = P.C; c->pk_used_rb = P.rb; c->pk_used_src = P.src; c->pk_used_threads = P.threads;
     return EF21_OK;
 }
 
@@ -543,8 +572,8 @@ ef21_status ef21_create(ef21_ctx** out, int32_t n, int64_t d, int32_t k, float g
     c->L = L;
     c->shards_loaded = false; c->inited = false; c->num_tiles = 0;
     c->path = EF21_PATH_AUTO; c->last_path = 0; c->launches = 0;
-    c->pk_cluster = 0; c->pk_rb = 0; c->pk_src = -1;
-    c->pk_used_cluster = c->pk_used_rb = 0; c->pk_used_src = -1;
+    c->pk_cluster = 0; c->pk_rb = 0; c->pk_src = -1; c->pk_threads = 0;
+    c->pk_used_cluster = c->pk_used_rb = 0; c->pk_used_src = -1; c->pk_used_threads = 0;
     c->spin_limit = 1u << 22;
     c->force_general_topk = false;
     c->aux_stream = nullptr; c->ev_fork = nullptr; c->ev_join = nullptr;
@@ -819,11 +848,19 @@ ef21_status ef21_set_path(ef21_ctx* c, int32_t path) {
 
 ef21_status ef21_set_persistent_shape(ef21_ctx* c, int32_t cluster_blocks, int32_t rows_per_batch, int32_t row_source) {
     if (!c || cluster_blocks < 0 || cluster_blocks > 8) return EF21_ERR_INVALID_ARG;
-    if (rows_per_batch != 0 && rows_per_batch != 8 && rows_per_batch != 16 && rows_per_batch != 32) return EF21_ERR_INVALID_ARG;
+    if (rows_per_batch != 0 && rows_per_batch != 4 && rows_per_batch != 8 && rows_per_batch != 16 && rows_per_batch != 32) return EF21_ERR_INVALID_ARG;
     if (row_source < -1 || row_source > 2) return EF21_ERR_INVALID_ARG;
     c->pk_cluster = cluster_blocks; c->pk_rb = rows_per_batch; c->pk_src = row_source;
     return EF21_OK;
 }
+
+ef21_status ef21_set_persistent_threads(ef21_ctx* c, int32_t threads_per_block) {
+    if (!c || (threads_per_block != 0 && threads_per_block != 256 && threads_per_block != 512)) return EF21_ERR_INVALID_ARG;
+    c->pk_threads = threads_per_block;
+    return EF21_OK;
+}
+
+int32_t ef21_get_persistent_threads(const ef21_ctx* c) { return c ? c->pk_used_threads : 0; }
 
 ef21_status ef21_get_persistent_shape(const ef21_ctx* c, int32_t* cluster_blocks, int32_t* rows_per_batch, int32_t* row_source) {
     if (!c) return EF21_ERR_INVALID_ARG;

@@ -33,8 +33,7 @@
 namespace ef21 {
 namespace cg = cooperative_groups;
 
-constexpr int PK_THREADS = 256;
-constexpr int PK_WARPS = PK_THREADS / 32;
+constexpr int PK_MAX_THREADS = 512;     // the kernel is instantiated for 256 and 512 threads per block
 constexpr int PK_MAX_K = 32;
 constexpr int PK_MAX_MSGS = 2048;       // n*k words staged in shared memory
 constexpr int PK_SCAN_MAX_MSGS = 128;   // up to this many messages every coordinate thread scans them all
@@ -135,10 +134,12 @@ __device__ __forceinline__ float comp_of(const float4& v, int c) {
     return c == 0 ? v.x : (c == 1 ? v.y : (c == 2 ? v.z : v.w));
 }
 
-template <int CHUNKS, int RB, int SRC>
-__global__ void __launch_bounds__(PK_THREADS, 1) persistent_kernel(const PersistParams p) {
-    constexpr int SH = (RB == 32) ? 0 : (RB == 16 ? 1 : 2);    // log2(32/RB)
-    static_assert(RB == 8 || RB == 16 || RB == 32, "RB");
+template <int CHUNKS, int RB, int SRC, int THREADS>
+__global__ void __launch_bounds__(THREADS, 1) persistent_kernel(const PersistParams p) {
+    constexpr int SH = (RB == 32) ? 0 : (RB == 16 ? 1 : (RB == 8 ? 2 : 3));    // log2(32/RB)
+    constexpr int WARPS = THREADS / 32;
+    static_assert(RB == 4 || RB == 8 || RB == 16 || RB == 32, "RB");
+    static_assert(THREADS == 256 || (THREADS == 512 && RB * CHUNKS <= 16), "512 threads leave 128 registers per thread");
     static_assert(RB * CHUNKS <= 32, "register budget");
     extern __shared__ __align__(16) unsigned char smem_raw[];
     cg::cluster_group cluster = cg::this_cluster();
@@ -155,8 +156,8 @@ __global__ void __launch_bounds__(PK_THREADS, 1) persistent_kernel(const Persist
     float* rterm = gs + ld;                                         // [ld] regulariser term at x
     float* gis = rterm + ld;                                        // [ld] g_i (leader block)
     float* vs = gis + ld;                                           // [ld] v = grad_i - g_i (leader block)
-    float* red = vs + ld;                                           // [PK_WARPS][ld]
-    float* part = red + PK_WARPS * ld;                              // [C][ld] (used in the leader)
+    float* red = vs + ld;                                           // [WARPS][ld]
+    float* part = red + WARPS * ld;                              // [C][ld] (used in the leader)
     unsigned long long* msg = reinterpret_cast<unsigned long long*>(part + C * ld);   // [nmsg]
     float* sacc = reinterpret_cast<float*>(msg + ((nmsg + 1) & ~1));                  // [ld] per-coordinate sum of messages
     unsigned char* touched = reinterpret_cast<unsigned char*>(sacc + ld);             // [ld] coordinate received a message
@@ -178,18 +179,18 @@ __global__ void __launch_bounds__(PK_THREADS, 1) persistent_kernel(const Persist
         mbar_init(&part_bar, 1u);
         fence_mbar_init_cluster();
     }
-    for (int j = tid; j < ld; j += PK_THREADS) { xs[j] = p.x[j]; gs[j] = p.g[j]; }
-    for (int j = tid; j < ld; j += PK_THREADS) { sacc[j] = 0.f; touched[j] = 0; }
+    for (int j = tid; j < ld; j += THREADS) { xs[j] = p.x[j]; gs[j] = p.g[j]; }
+    for (int j = tid; j < ld; j += THREADS) { sacc[j] = 0.f; touched[j] = 0; }
     if (SRC == PK_SRC_SMEM) {
         const float4* src = reinterpret_cast<const float4*>(p.A + r0 * (i64)ld);
         float4* dst = reinterpret_cast<float4*>(slice);
-        for (int e = tid; e < rows * chunks; e += PK_THREADS) dst[e] = src[e];
+        for (int e = tid; e < rows * chunks; e += THREADS) dst[e] = src[e];
     }
 
     // The leader block of the cluster keeps g_i in shared memory.
     const bool leader = crank == 0;
     if (leader)
-        for (int j = tid; j < ld; j += PK_THREADS) gis[j] = p.gi[(i64)worker * ld + j];
+        for (int j = tid; j < ld; j += THREADS) gis[j] = p.gi[(i64)worker * ld + j];
 
     // REG source: the (single) batch of this warp lives in registers for the whole kernel.
     float4 a[RB][CHUNKS];
@@ -213,7 +214,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) persistent_kernel(const Persist
         const int myrow = rb0 + (lane >> SH);
         y_reg = myrow < rows ? __ldg(p.y + r0 + myrow) : 0.f;
     };
-    if (SRC == PK_SRC_REG) load_batch(warp);     // host guarantees nbatch <= PK_WARPS
+    if (SRC == PK_SRC_REG) load_batch(warp);     // host guarantees nbatch <= WARPS
     if (C > 1) cluster.sync(); else __syncthreads();        // barriers initialised before any remote store
     const unsigned part_bytes = (unsigned)(C - 1) * (unsigned)chunks * 16u;
     const unsigned remote_part = map_to_rank(smem_u32(part), 0u), remote_bar = map_to_rank(smem_u32(&part_bar), 0u);
@@ -232,11 +233,11 @@ __global__ void __launch_bounds__(PK_THREADS, 1) persistent_kernel(const Persist
 
         if (!aborted) {
             // 1. x <- x - gamma g on this block's replica (Algorithm 2, first line of the loop)
-            for (int j = tid; j < ld; j += PK_THREADS) xs[j] = fmaf(-p.gamma, gs[j], xs[j]);
+            for (int j = tid; j < ld; j += THREADS) xs[j] = fmaf(-p.gamma, gs[j], xs[j]);
             if (leader && C > 1 && tid == 0) mbar_arrive_expect_tx(&part_bar, part_bytes);
             __syncthreads();
             if (leader)
-                for (int j = tid; j < ld; j += PK_THREADS) rterm[j] = regulariser_grad(p.lambda, xs[j]);
+                for (int j = tid; j < ld; j += THREADS) rterm[j] = regulariser_grad(p.lambda, xs[j]);
 
             // 2. partial gradient over this warp's batches
             float4 xr[CHUNKS], acc[CHUNKS];
@@ -246,7 +247,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) persistent_kernel(const Persist
                 xr[cs] = c < chunks ? reinterpret_cast<const float4*>(xs)[c] : make_float4(0.f, 0.f, 0.f, 0.f);
                 acc[cs] = make_float4(0.f, 0.f, 0.f, 0.f);
             }
-            for (int b = warp; b < nbatch; b += PK_WARPS) {
+            for (int b = warp; b < nbatch; b += WARPS) {
                 if (SRC != PK_SRC_REG) load_batch(b);
                 float pd[RB];
 #pragma unroll
@@ -274,10 +275,10 @@ __global__ void __launch_bounds__(PK_THREADS, 1) persistent_kernel(const Persist
 
             // 3. block partial (warps in ascending order) -> leader's shared memory.  Remote blocks send
             //    16-byte stores that credit the leader's barrier; they do not wait for anything.
-            for (int c = tid; c < chunks; c += PK_THREADS) {
+            for (int c = tid; c < chunks; c += THREADS) {
                 float4 sum = reinterpret_cast<const float4*>(red)[c];
 #pragma unroll
-                for (int w = 1; w < PK_WARPS; ++w) {
+                for (int w = 1; w < WARPS; ++w) {
                     const float4 o = reinterpret_cast<const float4*>(red + w * ld)[c];
                     sum.x = __fadd_rn(sum.x, o.x); sum.y = __fadd_rn(sum.y, o.y);
                     sum.z = __fadd_rn(sum.z, o.z); sum.w = __fadd_rn(sum.w, o.w);
@@ -308,7 +309,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) persistent_kernel(const Persist
             // 4. leader: gradient, difference, Top-k, state update, publish
             if (leader) {
                 const float mf = (float)m_i;
-                for (int j = tid; j < ld; j += PK_THREADS) {
+                for (int j = tid; j < ld; j += THREADS) {
                     float sum = part[j];
                     for (int cc = 1; cc < C; ++cc) sum = __fadd_rn(sum, part[cc * ld + j]);
                     const float grad = __fadd_rn(m_i > 0 ? __fdiv_rn(sum, mf) : 0.f, rterm[j]);
@@ -318,7 +319,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) persistent_kernel(const Persist
                 if (rank_select) {
                     // larger k: every coordinate counts the entries that precede it in (|v| descending, index
                     // ascending) order; the k entries of rank < k are the message
-                    for (int j = tid; j < ld; j += PK_THREADS) {
+                    for (int j = tid; j < ld; j += THREADS) {
                         unsigned char chosen = 0;
                         if (j < p.d) {
                             const unsigned kj = mag_key(vs[j]);
@@ -417,7 +418,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) persistent_kernel(const Persist
             }
 
             // 5. gather all n*k message words of this epoch (bounded spin)
-            for (int u = tid; u < nmsg; u += PK_THREADS) {
+            for (int u = tid; u < nmsg; u += THREADS) {
                 unsigned spins = 0;
                 unsigned long long w;
                 while (true) {
@@ -447,14 +448,14 @@ __global__ void __launch_bounds__(PK_THREADS, 1) persistent_kernel(const Persist
                 }
             }
             __syncthreads();
-            for (int j = tid; j < p.d; j += PK_THREADS)
+            for (int j = tid; j < p.d; j += THREADS)
                 if (touched[j]) {
                     gs[j] = __fadd_rn(gs[j], __fmul_rn(sacc[j], p.inv_n));
                     sacc[j] = 0.f; touched[j] = 0;
                 }
         } else if (!aborted) {
             // g_j += (1/n) * sum over workers (ascending) of the values sent for coordinate j
-            for (int j = tid; j < p.d; j += PK_THREADS) {
+            for (int j = tid; j < p.d; j += THREADS) {
                 float s = 0.f; bool touched = false;
 #pragma unroll 4
                 for (int u = 0; u < nmsg; ++u) {
@@ -473,9 +474,9 @@ __global__ void __launch_bounds__(PK_THREADS, 1) persistent_kernel(const Persist
         cluster.sync();
     }
     if (blockIdx.x == 0)
-        for (int j = tid; j < ld; j += PK_THREADS) { p.x[j] = xs[j]; p.g[j] = gs[j]; }
+        for (int j = tid; j < ld; j += THREADS) { p.x[j] = xs[j]; p.g[j] = gs[j]; }
     if (leader)
-        for (int j = tid; j < ld; j += PK_THREADS) p.gi[(i64)worker * ld + j] = gis[j];
+        for (int j = tid; j < ld; j += THREADS) p.gi[(i64)worker * ld + j] = gis[j];
 }
 
 // One-block self-check of the bounded wait: spins on a word that nobody writes and must come back

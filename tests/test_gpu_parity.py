@@ -302,6 +302,20 @@ def test_persistent_dimensions_and_ragged_shards(d, k, cluster, B, oracle32):
     assert h.poll() == 0
 
 
+@pytest.mark.parametrize("d,rb,threads,src", [(64, 4, 512, 1), (64, 16, 512, 0), (200, 8, 512, 2), (300, 4, 512, 1),
+                                              (300, 4, 256, 2), (120, 8, 512, 0), (500, 8, 256, 1)])
+def test_persistent_block_sizes(d, rb, threads, src, B, oracle32):
+    w = inputs.make_logistic("blocks", n=6, d=d, N=900, k=2, seed=1000 + d, features="gauss", flip=0.1, gamma=0.05, T=10)
+    h = make_gpu(w, path=2)
+    h.set_persistent_shape(2, rb, src)
+    h.set_persistent_threads(threads)
+    st = make_oracle_state(oracle32, w)
+    h.init(0); st.init(0)
+    assert lockstep(h, st, oracle32, w, 10) <= 1
+    assert h.get_persistent_shape() == (2, rb, src) and h.get_persistent_threads() == threads
+    assert h.poll() == 0
+
+
 def test_persistent_many_steps_in_one_launch_equals_single_steps(B):
     w = inputs.config(1)
     a = make_gpu(w, path=2); a.init(0); a.step(300)
