@@ -72,7 +72,7 @@ enum {
 enum {
     EF21_PATH_AUTO = 0,       /* pick the fastest path that supports the shape */
     EF21_PATH_LAUNCHES = 1,   /* one kernel launch per stage, any shape */
-    EF21_PATH_PERSISTENT = 2  /* one cooperative kernel for all steps; shards on chip */
+    EF21_PATH_PERSISTENT = 2  /* one cluster kernel for all steps; shards on chip */
 };
 
 const char* ef21_status_string(ef21_status s);

@@ -512,18 +512,13 @@ ef21_status run_persistent(ef21_ctx* c, const PersistPlan& P, int steps) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(c->n * P.C)); cfg.blockDim = dim3((unsigned)P.threads); cfg.dynamicSmemBytes = P.smem;
     cfg.stream = c->stream;
-    cudaLaunchAttribute attr[2];
+    // A plain cluster launch: that all n clusters fit on the device at once was checked with the
+    // occupancy query when the plan was made.
+    cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = (unsigned)P.C; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    attr[1].id = cudaLaunchAttributeCooperative;
-    attr[1].val.cooperative = 1;
-    cfg.attrs = attr; cfg.numAttrs = 2;
+    cfg.attrs = attr; cfg.numAttrs = 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, P.kernel, p);
-    if (e != cudaSuccess) {           // residency was already checked; retry as a plain cluster launch
-        cudaGetLastError();
-        cfg.numAttrs = 1;
-        e = cudaLaunchKernelEx(&cfg, P.kernel, p);
-    }
     if (e != cudaSuccess) { cudaGetLastError(); return EF21_ERR_CUDA; }
     c->launches += 1;
     c->pk_used_cluster = P.C; c->pk_used_rb = P.rb; c->pk_used_src = P.src; c->pk_used_threads = P.threads;

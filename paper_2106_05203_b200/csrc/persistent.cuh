@@ -174,6 +174,11 @@ __global__ void __launch_bounds__(THREADS, 1) persistent_kernel(const PersistPar
     const int rows = (int)(r1 - r0);
     const int nbatch = (rows + RB - 1) / RB;
 
+    // The launch must really have put C blocks into each cluster; otherwise nobody would send partials.
+    if ((int)cluster.num_blocks() != C) {
+        if (tid == 0) record_error(p.status, 7u /* EF21_ERR_UNSUPPORTED */);
+        return;
+    }
     if (tid == 0) {
         abort_flag = 0;
         mbar_init(&part_bar, 1u);
