@@ -169,6 +169,30 @@ class State:
                                     _c_int64(self.k), _p(V), self.o._creal(self.gamma),
                                     *self._args_state())
 
+    # -- EF21+ (Algorithm 3) -------------------------------------------------
+    def _choice(self):
+        if not hasattr(self, "choice"):
+            self.choice = np.zeros(self.n, dtype=np.int32)
+        return self.choice
+
+    def plus_step(self, steps: int = 1) -> None:
+        ch = self._choice()
+        self.o.lib.ef21o_plus_step(_c_int32(steps), _c_int32(self.n), _c_int64(self.d), _c_int64(self.k),
+                                   _p(self.A), _p(self.y), _p(self.off), _c_double(self.lam),
+                                   self.o._creal(self.gamma), *self._args_state(), _p(ch))
+
+    def plus_step_grads(self, V, steps: int = 1) -> None:
+        V = self.o._r(V)
+        ch = self._choice()
+        self.o.lib.ef21o_plus_step_grads(_c_int32(steps), _c_int32(self.n), _c_int64(self.d), _c_int64(self.k),
+                                         _p(V), self.o._creal(self.gamma), *self._args_state(), _p(ch))
+
+    def plus_round(self, grads) -> None:
+        grads = self.o._r(grads)
+        ch = self._choice()
+        self.o.lib.ef21o_plus_round(_c_int32(self.n), _c_int64(self.d), _c_int64(self.k), _p(grads),
+                                    _p(self.gi), _p(self.g), _p(self.idx), _p(self.val), _p(ch))
+
     def round(self, grads) -> None:
         """One message round (no x update) given the local gradients."""
         grads = self.o._r(grads)

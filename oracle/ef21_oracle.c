@@ -282,3 +282,75 @@ void ef21o_step_grads(int32_t steps, int32_t n, int64_t d, int64_t k, const real
         ef21o_round(n, d, k, V, gi, g, idx, val);
     }
 }
+
+/* ------------------------------------------------------------------ */
+/* EF21+ (Algorithm 3): per node the better of C and the Markov compressor */
+/* ------------------------------------------------------------------ */
+
+/* One round of Algorithm 3 given the local gradients: for every worker
+ *     m_i = g_i + C(grad_i - g_i)        (Markov compressor)
+ *     b_i = C(grad_i)                    (plain compressor)
+ *     M_i = ||m_i - grad_i||^2,  B_i = ||b_i - grad_i||^2      (fp64 sums over the stored vectors)
+ *     g_i <- m_i if M_i <= B_i else b_i
+ * and the master's g = (1/n) sum_i g_i (sum over ascending i, then one multiply by 1/n).
+ * idx/val receive the compressed vector that was used (C(grad_i - g_i) or C(grad_i)),
+ * choice[i] = 0 for the Markov branch, 1 for the plain one. */
+void ef21o_plus_round(int32_t n, int64_t d, int64_t k, const real* grads, real* gi, real* g,
+                      int32_t* idx, real* val, int32_t* choice) {
+    real* v = (real*)malloc((size_t)d * sizeof(real));
+    real* m = (real*)malloc((size_t)d * sizeof(real));
+    int32_t* ib = (int32_t*)malloc((size_t)k * sizeof(int32_t));
+    real* vb = (real*)malloc((size_t)k * sizeof(real));
+    unsigned char* inb = (unsigned char*)malloc((size_t)d);
+    for (int32_t i = 0; i < n; ++i) {
+        const real* gr = grads + (int64_t)i * d;
+        real* gs = gi + (int64_t)i * d;
+        int32_t* im = idx + (int64_t)i * k;
+        real* vm = val + (int64_t)i * k;
+        for (int64_t j = 0; j < d; ++j) { v[j] = gr[j] - gs[j]; m[j] = gs[j]; }
+        ef21o_topk(v, d, k, im, vm);
+        for (int64_t t = 0; t < k; ++t) m[im[t]] = m[im[t]] + vm[t];
+        double M = 0.0;
+        for (int64_t j = 0; j < d; ++j) { double e = (double)m[j] - (double)gr[j]; M += e * e; }
+        ef21o_topk(gr, d, k, ib, vb);
+        memset(inb, 0, (size_t)d);
+        for (int64_t t = 0; t < k; ++t) inb[ib[t]] = 1;
+        double B = 0.0;
+        for (int64_t j = 0; j < d; ++j) if (!inb[j]) { double e = (double)gr[j]; B += e * e; }
+        if (M <= B) {
+            memcpy(gs, m, (size_t)d * sizeof(real));
+            choice[i] = 0;
+        } else {
+            for (int64_t j = 0; j < d; ++j) gs[j] = (real)0;
+            for (int64_t t = 0; t < k; ++t) { gs[ib[t]] = vb[t]; im[t] = ib[t]; vm[t] = vb[t]; }
+            choice[i] = 1;
+        }
+    }
+    const real inv_n = (real)1 / (real)n;
+    for (int64_t j = 0; j < d; ++j) {
+        real s = (real)0;
+        for (int32_t i = 0; i < n; ++i) s = s + gi[(int64_t)i * d + j];
+        g[j] = s * inv_n;
+    }
+    free(v); free(m); free(ib); free(vb); free(inb);
+}
+
+void ef21o_plus_step(int32_t steps, int32_t n, int64_t d, int64_t k, const float* A, const float* y,
+                     const int64_t* row_off, double lam, real gamma,
+                     real* x, real* gi, real* g, int32_t* idx, real* val, int32_t* choice) {
+    real* grads = (real*)malloc((size_t)n * (size_t)d * sizeof(real));
+    for (int32_t t = 0; t < steps; ++t) {
+        ef21o_x_update(d, gamma, g, x);
+        ef21o_all_grads(n, d, A, y, row_off, x, lam, grads);
+        ef21o_plus_round(n, d, k, grads, gi, g, idx, val, choice);
+    }
+    free(grads);
+}
+
+void ef21o_plus_step_grads(int32_t steps, int32_t n, int64_t d, int64_t k, const real* V, real gamma,
+                           real* x, real* gi, real* g, int32_t* idx, real* val, int32_t* choice) {
+    for (int32_t t = 0; t < steps; ++t) {
+        ef21o_x_update(d, gamma, g, x);
+        ef21o_plus_round(n, d, k, V, gi, g, idx, val, choice);
+    }
+}

@@ -387,3 +387,79 @@ def test_fp32_state_updates_are_single_rounded_operations(oracle32):
         g_expect = np.where(touched, (g + (s * inv_n).astype(np.float32)).astype(np.float32), g)
         np.testing.assert_array_equal(st.gi, gi)
         np.testing.assert_array_equal(st.g, g_expect)
+
+
+# ---------------------------------------------------------------------------
+# EF21+ (Algorithm 3)
+# ---------------------------------------------------------------------------
+
+def _read_kv(path):
+    out = {}
+    with open(path) as fh:
+        for line in fh:
+            tok = line.split()
+            if tok and not tok[0].startswith("#"):
+                out[tok[0]] = [float(t) for t in tok[1:]]
+    return out
+
+
+@pytest.mark.parametrize("precision", ["f32", "f64"])
+def test_alg3_hand_worked_round(precision):
+    o = oracle_mod.Oracle(precision)
+    kv = _read_kv(os.path.join(GOLDEN, "alg3_hand_example.txt"))
+    st = oracle_mod.State(o, 2, 2, 1, 0.5)
+    st.gi[:] = np.array([kv["g1"], kv["g2"]])
+    st.plus_round(np.array([kv["grad1"], kv["grad2"]]))
+    np.testing.assert_array_equal(st.gi, [kv["new_g1"], kv["new_g2"]])
+    np.testing.assert_array_equal(st.g, kv["new_g"])
+    np.testing.assert_array_equal(st.choice, kv["choice"])
+    np.testing.assert_array_equal(st.idx[:, 0], kv["idx"])
+    np.testing.assert_array_equal(st.val[:, 0], kv["val"])
+
+
+def test_ef21_plus_takes_the_better_compressor_and_keeps_the_rate(oracle64):
+    # Section 3.4: G_i^{t+1} <= min(B_i, M_i) <= M_i, so Lemma 2's bound and Theorem 1 carry over;
+    # g is the plain mean of the g_i (Algorithm 3, master line).
+    w = inputs.config(0)
+    k = 4
+    gamma = inputs.theory_gamma(w.A, w.row_offsets, w.lam, k)
+    theta = 1 - math.sqrt(1 - k / w.d)
+    st = oracle_mod.State(oracle64, w.n, w.d, k, gamma, w.lam, w.A, w.y, w.row_offsets, w.x0)
+    st.init(0)
+    T = 40
+    f0 = st.loss()
+    _, G0 = oracle64.diagnostics(w.A, w.y, w.row_offsets, st.x, w.lam, st.gi)
+    sq = []
+    took_plain = 0
+    for _ in range(T):
+        nrm2, _ = oracle64.diagnostics(w.A, w.y, w.row_offsets, st.x, w.lam, st.gi)
+        sq.append(nrm2)
+        gi_old = st.gi.copy()
+        st.plus_step(1)
+        grads = st.grads()
+        np.testing.assert_allclose(st.g, st.gi.mean(axis=0), rtol=0, atol=1e-15)
+        for i in range(w.n):
+            ib, vb = _brute_topk(grads[i], k)
+            b = np.zeros(w.d); b[ib] = vb
+            im, vm = _brute_topk(grads[i] - gi_old[i], k)
+            m = gi_old[i].copy(); m[im] += vm
+            B, M = np.sum((b - grads[i]) ** 2), np.sum((m - grads[i]) ** 2)
+            expect = m if M <= B else b
+            np.testing.assert_allclose(st.gi[i], expect, rtol=0, atol=1e-15)
+            assert st.choice[i] == (0 if M <= B else 1)
+            assert np.sum((st.gi[i] - grads[i]) ** 2) <= min(B, M) * (1 + 1e-12) + 1e-30
+            took_plain += int(st.choice[i])
+    assert np.mean(sq) <= 2 * f0 / (gamma * T) + G0 / (theta * T)
+
+
+def test_ef21_plus_plain_branch_is_exercised(oracle64):
+    # far-off g_i (arbitrary initialisation is allowed, Section 3.3) make C(grad) the better choice at first
+    w = inputs.config(0)
+    st = oracle_mod.State(oracle64, w.n, w.d, 4, 0.05, w.lam, w.A, w.y, w.row_offsets, w.x0)
+    st.init(1)
+    st.gi[:] = 3.0
+    st.g[:] = 3.0
+    st.plus_step(1)
+    assert st.choice.sum() == w.n
+    for i in range(w.n):
+        assert np.count_nonzero(st.gi[i]) <= 4
