@@ -231,8 +231,9 @@ def run_ours(args):
             dist.destroy_process_group()
         return
 
-    def time_logistic(w, k, steps, warmup, repeats=3, with_clocks=False):
+    def time_logistic(w, k, steps, warmup, repeats=3, with_clocks=False, variant=0):
         h = B.EF21(w.n, w.d, k, w.gamma, w.lam, total_rows=w.N, device=device)
+        h.set_variant(variant)
         h.load_shards(dev(w.A), dev(w.y), w.row_offsets)
         h.init(B.INIT_COMPRESSED)
         x0, g0, gi0, _, _ = h.get_state()
@@ -339,6 +340,11 @@ def run_ours(args):
                            "us_per_iteration": rr["ms"] / wk.T * 1e3, "algorithmic_GBps": gbs, "frac_of_hbm_peak": gbs / peak,
                            "launches": rr["launches"], "persistent_shape": rr["shape"], "f_end": rr["f_end"]})
         others.append(time_stress(None, 50, 3))
+        # EF21+ (Algorithm 3) on the headline shapes: launch-per-stage kernels, two Top-k per worker and step
+        wp = inputs.config(HEADLINE)
+        rp = time_logistic(wp, wp.k, 500, 10, variant=B.VARIANT_EF21_PLUS)
+        others.append({"workload": f"EF21+ on configs[{HEADLINE}] {wp.name} Top-{wp.k}", "iterations_per_s": 500 / (rp["ms"] * 1e-3),
+                       "us_per_iteration": rp["ms"] / 500 * 1e3, "launches": rp["launches"], "f_end": rp["f_end"]})
         line["workloads"] = others
 
     if world > 1:

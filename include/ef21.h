@@ -75,6 +75,12 @@ enum {
     EF21_PATH_PERSISTENT = 2  /* one cluster kernel for all steps; shards on chip */
 };
 
+/* Which method ef21_step / ef21_step_grads run. */
+enum {
+    EF21_VARIANT_EF21 = 0,      /* Algorithm 2 */
+    EF21_VARIANT_EF21_PLUS = 1  /* Algorithm 3: per worker the better of C and the Markov compressor */
+};
+
 const char* ef21_status_string(ef21_status s);
 
 /* Bytes of device workspace ef21_create needs for n workers, dimension d, k kept
@@ -174,6 +180,17 @@ ef21_status ef21_eval(ef21_ctx* ctx, double* f, double* grad_norm2, double* G);
 /* Synchronises the stream and returns the device status word: EF21_OK, or the first
  * error a kernel recorded (EF21_ERR_TIMEOUT, EF21_ERR_NONFINITE), or EF21_ERR_CUDA. */
 ef21_status ef21_poll(ef21_ctx* ctx);
+
+/* EF21+ (Section 3.4, Algorithm 3).  With EF21_VARIANT_EF21_PLUS every step computes, per worker,
+ * b_i = C(grad f_i(x)) and m_i = g_i + C(grad f_i(x) - g_i), the distortions B_i = ||b_i - grad f_i(x)||^2
+ * and M_i = ||m_i - grad f_i(x)||^2 (fp64 sums of the fp32 vectors), sets g_i = m_i if M_i <= B_i and
+ * g_i = b_i otherwise, and recomputes g = (1/n) sum_i g_i (ascending i, then one multiply).  Runs on
+ * the launch path only (EF21_PATH_PERSISTENT returns EF21_ERR_UNSUPPORTED).  The "last message" of
+ * ef21_get_state is the compressed vector that was used.  Initialisation is that of Algorithm 2. */
+ef21_status ef21_set_variant(ef21_ctx* ctx, int32_t variant);
+/* choice_host[n]: 0 where the last EF21+ step kept the Markov compressor, 1 where it took C(grad);
+ * synchronises. */
+ef21_status ef21_get_plus_choice(ef21_ctx* ctx, int32_t* choice_host);
 
 /* Top-k algorithm used inside the EF21 rounds of the launch path: 0 = automatic (long vectors,
  * d >= 2^18 and k <= 6144, take the one-pass path: sampled threshold, single streaming pass,

@@ -22,6 +22,7 @@ STATUS_NAMES = {0: "EF21_OK", 1: "EF21_ERR_INVALID_ARG", 2: "EF21_ERR_STATE", 3:
                 4: "EF21_ERR_CUDA", 5: "EF21_ERR_TIMEOUT", 6: "EF21_ERR_NONFINITE", 7: "EF21_ERR_UNSUPPORTED"}
 INIT_COMPRESSED, INIT_ZERO, INIT_GRADIENT = 0, 1, 2
 PATH_AUTO, PATH_LAUNCHES, PATH_PERSISTENT = 0, 1, 2
+VARIANT_EF21, VARIANT_EF21_PLUS = 0, 1
 
 # name -> (restype, argtypes); mirrors include/ef21.h
 _i32, _i64, _f32, _sz, _vp = ctypes.c_int32, ctypes.c_int64, ctypes.c_float, ctypes.c_size_t, ctypes.c_void_p
@@ -47,6 +48,8 @@ SIGNATURES = {
     "ef21_set_state": (ctypes.c_int, [_vp, _vp, _vp, _vp]),
     "ef21_eval": (ctypes.c_int, [_vp, _dp, _dp, _dp]),
     "ef21_poll": (ctypes.c_int, [_vp]),
+    "ef21_set_variant": (ctypes.c_int, [_vp, _i32]),
+    "ef21_get_plus_choice": (ctypes.c_int, [_vp, _vp]),
     "ef21_set_topk_algorithm": (ctypes.c_int, [_vp, _i32]),
     "ef21_fallback_count": (ctypes.c_int, [_vp, ctypes.POINTER(_i64)]),
     "ef21_clear_status": (ctypes.c_int, [_vp]),
@@ -229,6 +232,14 @@ class EF21:
 
     def poll(self) -> int:
         return int(_lib.ef21_poll(self._h))
+
+    def set_variant(self, variant: int) -> None:
+        _check(_lib.ef21_set_variant(self._h, variant), "ef21_set_variant")
+
+    def get_plus_choice(self) -> np.ndarray:
+        out = np.zeros(self.n, dtype=np.int32)
+        _check(_lib.ef21_get_plus_choice(self._h, _np_ptr(out)), "ef21_get_plus_choice")
+        return out
 
     def set_topk_algorithm(self, algorithm: int) -> None:
         _check(_lib.ef21_set_topk_algorithm(self._h, algorithm), "ef21_set_topk_algorithm")

@@ -12,6 +12,7 @@
 #include "common.cuh"
 #include "grad.cuh"
 #include "persistent.cuh"
+#include "plus.cuh"
 #include "stress.cuh"
 #include "topk.cuh"
 
@@ -75,6 +76,7 @@ struct Layout {
     int tile_rows;     // rows per gradient tile
     i64 max_tiles;     // capacity of the gradient tile table
     size_t status, x, g, gi, msg_idx, msg_val, topk, agg_off, eval_out, slots;
+    size_t msg2_idx, msg2_val, plus_old, plus_choice, plus_bitmap;    // EF21+ (Algorithm 3)
     size_t A, y, row_off, tile_begin, tiles, partial, loss_partial, grad;
     size_t total;
     TopkLayout tk;
@@ -97,6 +99,11 @@ Layout make_layout(i64 n, i64 d, i64 k, i64 N) {
     L.agg_off = take((size_t)n * (L.agg_tiles + 1) * 4);
     L.eval_out = take(256);
     L.slots = take((size_t)2 * n * k * 8);
+    L.msg2_idx = take((size_t)n * k * 4);
+    L.msg2_val = take((size_t)n * k * 4);
+    L.plus_old = take((size_t)n * k * 4);
+    L.plus_choice = take((size_t)n * 4);
+    L.plus_bitmap = take((size_t)n * ((d + 31) / 32) * 4);
     L.tile_rows = 0; L.max_tiles = 0;
     L.A = L.y = L.row_off = L.tile_begin = L.tiles = L.partial = L.loss_partial = L.grad = 0;
     if (N > 0) {
@@ -133,6 +140,7 @@ struct ef21_ctx {
     int pk_used_cluster, pk_used_rb, pk_used_src, pk_used_threads;
     unsigned spin_limit;
     bool force_general_topk;
+    int variant;                        // EF21_VARIANT_*
     cudaStream_t aux_stream;            // created on first use: overlaps the next threshold estimate
     cudaEvent_t ev_fork, ev_join;
     i64 launches;
@@ -294,6 +302,31 @@ ef21_status enqueue_round_aggregate(ef21_ctx* c, bool update_x) {
 ef21_status enqueue_round(ef21_ctx* c, const float* a, i64 pitch_a, bool update_x) {
     EF(enqueue_round_select(c, a, pitch_a, false));
     return enqueue_round_aggregate(c, update_x);
+}
+
+// One round of EF21+ (Algorithm 3) on local gradients a: both compressed vectors, the choice by
+// distortion, g_i <- chosen, g = (1/n) sum g_i.
+ef21_status enqueue_plus_round(ef21_ctx* c, const float* a, i64 pitch_a) {
+    TopkBuffers B = topk_buffers(c->ws + c->L.topk, c->L.tk);
+    int* idx_b = c->at<int>(c->L.msg2_idx);
+    float* val_b = c->at<float>(c->L.msg2_val);
+    if (B.fast && !c->force_general_topk) {
+        EF(enqueue_topk_fast(c->stream, a, pitch_a, c->gi(), c->L.ld, c->n, c->d, c->k, c->msg_idx(), c->msg_val(),
+                             nullptr, 0, B, &c->launches));
+        EF(enqueue_topk_fast(c->stream, a, pitch_a, nullptr, 0, c->n, c->d, c->k, idx_b, val_b, nullptr, 0, B, &c->launches));
+    } else {
+        EF(enqueue_topk_general(c->stream, a, pitch_a, c->gi(), c->L.ld, c->n, c->d, c->k, c->msg_idx(), c->msg_val(), B,
+                                &c->launches));
+        EF(enqueue_topk_general(c->stream, a, pitch_a, nullptr, 0, c->n, c->d, c->k, idx_b, val_b, B, &c->launches));
+    }
+    plus_choose_kernel<<<c->n, PLUS_BLOCK, 0, c->stream>>>(a, pitch_a, c->gi(), c->L.ld, c->d, c->k, c->msg_idx(), c->msg_val(),
+                                                          idx_b, val_b, c->at<float>(c->L.plus_old), c->at<unsigned>(c->L.plus_bitmap),
+                                                          c->at<int>(c->L.plus_choice));
+    const unsigned blocks = (unsigned)std::min<i64>(ceil_div(c->d, 256), 148 * 8);
+    dense_mean_kernel<<<blocks, 256, 0, c->stream>>>(c->gi(), c->L.ld, c->n, c->d, 1.0f / (float)c->n, c->g());
+    c->launches += 2;
+    CU(cudaGetLastError());
+    return EF21_OK;
 }
 
 ef21_status enqueue_x_update(ef21_ctx* c) {
@@ -571,6 +604,7 @@ ef21_status ef21_create(ef21_ctx** out, int32_t n, int64_t d, int32_t k, float g
     c->pk_used_cluster = c->pk_used_rb = 0; c->pk_used_src = -1; c->pk_used_threads = 0;
     c->spin_limit = 1u << 22;
     c->force_general_topk = false;
+    c->variant = EF21_VARIANT_EF21;
     c->aux_stream = nullptr; c->ev_fork = nullptr; c->ev_join = nullptr;
     cudaError_t e = cudaMemsetAsync(c->ws + L.status, 0, 256, c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->x(), 0, (size_t)L.ld * 4, c->stream);
@@ -579,6 +613,7 @@ ef21_status ef21_create(ef21_ctx** out, int32_t n, int64_t d, int32_t k, float g
     if (e == cudaSuccess) e = cudaMemsetAsync(c->msg_idx(), 0, (size_t)n * k * 4, c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->msg_val(), 0, (size_t)n * k * 4, c->stream);
     if (e == cudaSuccess && L.tk.fast) e = cudaMemsetAsync(c->ws + L.topk + L.tk.slow_count, 0, 4, c->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->ws + L.plus_choice, 0, (size_t)n * 4, c->stream);
     if (e != cudaSuccess) { delete c; return EF21_ERR_CUDA; }
     *out = c;
     return EF21_OK;
@@ -644,6 +679,16 @@ ef21_status ef21_step(ef21_ctx* c, int32_t steps) {
     if (!c || steps < 0) return EF21_ERR_INVALID_ARG;
     if (!c->shards_loaded || !c->inited) return EF21_ERR_STATE;
     if (steps == 0) return EF21_OK;
+    if (c->variant == EF21_VARIANT_EF21_PLUS) {
+        if (c->path == EF21_PATH_PERSISTENT) return EF21_ERR_UNSUPPORTED;
+        for (int t = 0; t < steps; ++t) {
+            EF(enqueue_x_update(c));
+            EF(enqueue_grads(c, false));
+            EF(enqueue_plus_round(c, c->at<float>(c->L.grad), c->L.ld));
+        }
+        c->last_path = EF21_PATH_LAUNCHES;
+        return EF21_OK;
+    }
     if (c->path != EF21_PATH_LAUNCHES) {
         PersistPlan P = plan_persistent(c);
         if (P.ok) {
@@ -665,6 +710,14 @@ ef21_status ef21_step(ef21_ctx* c, int32_t steps) {
 ef21_status ef21_step_grads(ef21_ctx* c, const float* V_dev, int32_t steps) {
     if (!c || !V_dev || steps < 0) return EF21_ERR_INVALID_ARG;
     if (!c->inited) return EF21_ERR_STATE;
+    if (c->variant == EF21_VARIANT_EF21_PLUS) {
+        for (int t = 0; t < steps; ++t) {
+            EF(enqueue_x_update(c));
+            EF(enqueue_plus_round(c, V_dev, c->d));
+        }
+        c->last_path = EF21_PATH_LAUNCHES;
+        return EF21_OK;
+    }
     const bool fast = c->L.tk.fast && !c->force_general_topk;
     if (fast && steps > 1 && !c->aux_stream) {
         // V is the same at every step, so the threshold estimate of step t+1 only waits for the
@@ -862,6 +915,19 @@ ef21_status ef21_get_persistent_shape(const ef21_ctx* c, int32_t* cluster_blocks
     if (cluster_blocks) *cluster_blocks = c->pk_used_cluster;
     if (rows_per_batch) *rows_per_batch = c->pk_used_rb;
     if (row_source) *row_source = c->pk_used_src;
+    return EF21_OK;
+}
+
+ef21_status ef21_set_variant(ef21_ctx* c, int32_t variant) {
+    if (!c || (variant != EF21_VARIANT_EF21 && variant != EF21_VARIANT_EF21_PLUS)) return EF21_ERR_INVALID_ARG;
+    c->variant = variant;
+    return EF21_OK;
+}
+
+ef21_status ef21_get_plus_choice(ef21_ctx* c, int32_t* choice_host) {
+    if (!c || !choice_host) return EF21_ERR_INVALID_ARG;
+    CU(cudaMemcpyAsync(choice_host, c->at<int>(c->L.plus_choice), (size_t)c->n * 4, cudaMemcpyDeviceToHost, c->stream));
+    CU(cudaStreamSynchronize(c->stream));
     return EF21_OK;
 }
 

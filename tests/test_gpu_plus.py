@@ -1,0 +1,95 @@
+"""GPU parity for EF21+ (Algorithm 3): the choice between the plain and the Markov compressor, the
+resulting worker states and the recomputed average, against the oracle."""
+import os
+
+import numpy as np
+import pytest
+
+import ef21_inputs as inputs
+import oracle as oracle_mod
+from gpu_util import dev, make_gpu, make_oracle_state, rel_l2, set_gpu_state_from_oracle
+
+pytestmark = pytest.mark.gpu
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2106_05203_b200 import binding
+    return binding
+
+
+def _assert_bitwise(h, st, what):
+    x, g, gi, li, lv = h.get_state_host()
+    np.testing.assert_array_equal(h.get_plus_choice(), st.choice, err_msg=f"{what}: choice")
+    np.testing.assert_array_equal(li, st.idx, err_msg=f"{what}: idx")
+    np.testing.assert_array_equal(lv.view(np.uint32), st.val.view(np.uint32), err_msg=f"{what}: val")
+    np.testing.assert_array_equal(gi.view(np.uint32), st.gi.view(np.uint32), err_msg=f"{what}: g_i")
+    np.testing.assert_array_equal(g.view(np.uint32), st.g.view(np.uint32), err_msg=f"{what}: g")
+    np.testing.assert_array_equal(x.view(np.uint32), st.x.view(np.uint32), err_msg=f"{what}: x")
+
+
+def test_hand_worked_round_on_gpu(B):
+    from test_oracle_pins import _read_kv
+    kv = _read_kv(os.path.join(GOLDEN, "alg3_hand_example.txt"))
+    h = B.EF21(2, 2, 1, 0.5)
+    h.set_variant(B.VARIANT_EF21_PLUS)
+    h.set_state(dev(np.zeros(2, np.float32)), dev(np.zeros(2, np.float32)),
+                dev(np.array([kv["g1"], kv["g2"]], dtype=np.float32)))
+    h.step_grads(dev(np.array([kv["grad1"], kv["grad2"]], dtype=np.float32)), 1)
+    x, g, gi, li, lv = h.get_state_host()
+    np.testing.assert_array_equal(gi, [kv["new_g1"], kv["new_g2"]])
+    np.testing.assert_array_equal(g, kv["new_g"])
+    np.testing.assert_array_equal(h.get_plus_choice(), kv["choice"])
+    np.testing.assert_array_equal(li[:, 0], kv["idx"])
+    np.testing.assert_array_equal(lv[:, 0], kv["val"])
+
+
+@pytest.mark.parametrize("n,d,k", [(5, 300, 7), (3, 5000, 40), (4, 300000, 300)])
+def test_supplied_gradients_both_branches_bit_exact(n, d, k, B, oracle32):
+    # a changing gradient sequence with jumps: some rounds keep the Markov compressor, others restart from C(grad)
+    rng = np.random.default_rng(d)
+    h = B.EF21(n, d, k, 0.05); h.set_variant(B.VARIANT_EF21_PLUS)
+    st = oracle_mod.State(oracle32, n, d, k, 0.05)
+    h.init_grads(None, 1); st.init(1)
+    base = rng.standard_normal((n, d)).astype(np.float32)
+    seen = set()
+    for t in range(8):
+        scale = np.float32(1.0 if t % 3 else 25.0)
+        V = (base * scale + 0.01 * rng.standard_normal((n, d))).astype(np.float32)
+        h.step_grads(dev(V), 1); st.plus_step_grads(V, 1)
+        _assert_bitwise(h, st, f"step {t}")
+        seen |= set(st.choice.tolist())
+    assert seen == {0, 1}
+    assert h.poll() == 0
+
+
+def test_logistic_ef21_plus_tracks_the_oracle(B, oracle32):
+    w = inputs.config(0)
+    h = make_gpu(w); h.set_variant(B.VARIANT_EF21_PLUS)
+    st = make_oracle_state(oracle32, w)
+    h.init(0); st.init(0)
+    for t in range(30):
+        h.step(1); st.plus_step(1)
+        x, g, gi, li, lv = h.get_state_host()
+        np.testing.assert_array_equal(h.get_plus_choice(), st.choice)
+        np.testing.assert_array_equal(li, st.idx)
+        assert rel_l2(x, st.x) <= 1e-4 or np.linalg.norm(st.x) == 0
+        assert np.max(np.abs(gi - st.gi)) <= 1e-5 * np.max(np.abs(st.gi))
+        set_gpu_state_from_oracle(h, st)
+    assert h.last_path == B.PATH_LAUNCHES
+    h.set_path(B.PATH_PERSISTENT)
+    with pytest.raises(B.Ef21Error) as e:
+        h.step(1)
+    assert e.value.status == 7
+
+
+def test_free_running_ef21_plus_paper_shape(B, oracle32):
+    w = inputs.config(1)
+    h = make_gpu(w); h.set_variant(B.VARIANT_EF21_PLUS)
+    st = make_oracle_state(oracle32, w)
+    h.init(0); st.init(0)
+    h.step(60); st.plus_step(60)
+    x = h.get_state_host()[0]
+    assert rel_l2(x, st.x) <= 1e-4
+    assert h.eval()[0] == pytest.approx(st.loss(), rel=1e-4)
