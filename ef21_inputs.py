@@ -89,7 +89,7 @@ def _planted_labels(rng: np.random.Generator, A: np.ndarray, w: np.ndarray, flip
     return y.astype(np.float32)
 
 
-def smoothness_constants(A: np.ndarray, row_offsets: np.ndarray, lam: float) -> np.ndarray:
+def smoothness_constants(A: np.ndarray, row_offsets: np.ndarray, lam: float, objective: str = "logistic") -> np.ndarray:
     """Upper bounds L_i on the gradient-Lipschitz constants of the local losses.
 
     For the logistic term the curvature of log(1+exp(-t)) is at most 1/4, so the
@@ -106,13 +106,14 @@ def smoothness_constants(A: np.ndarray, row_offsets: np.ndarray, lam: float) -> 
             L[i] = 2.0 * lam
             continue
         gram = Ai.T @ Ai
-        L[i] = float(np.linalg.eigvalsh(gram)[-1]) / (4.0 * m) + 2.0 * lam
+        curvature = 0.25 if objective == "logistic" else 2.0      # second derivative bound of the loss in the margin
+        L[i] = curvature * float(np.linalg.eigvalsh(gram)[-1]) / m + 2.0 * lam
     return L
 
 
-def gamma_one_over_L(A: np.ndarray, row_offsets: np.ndarray, lam: float) -> float:
+def gamma_one_over_L(A: np.ndarray, row_offsets: np.ndarray, lam: float, objective: str = "logistic") -> float:
     """gamma = 1/L with L = mean_i L_i (the bound L <= (1/n) sum L_i of Section 3.3)."""
-    L = smoothness_constants(A, row_offsets, lam)
+    L = smoothness_constants(A, row_offsets, lam, objective)
     return float(np.float32(1.0 / float(np.mean(L))))
 
 

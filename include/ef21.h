@@ -75,6 +75,13 @@ enum {
     EF21_PATH_PERSISTENT = 2  /* one cluster kernel for all steps; shards on chip */
 };
 
+/* Local objective f_i on worker i's rows (a_r, y_r); both get the regulariser lambda sum_j x_j^2/(1+x_j^2)
+ * added (pass lambda = 0 for none). */
+enum {
+    EF21_OBJECTIVE_LOGISTIC = 0,      /* (1/m_i) sum_r log(1 + exp(-y_r a_r.x))   (Section 5, Eq. 19) */
+    EF21_OBJECTIVE_LEAST_SQUARES = 1  /* (1/m_i) sum_r (a_r.x - y_r)^2            (Appendix A.2, least squares) */
+};
+
 /* Which method ef21_step / ef21_step_grads run. */
 enum {
     EF21_VARIANT_EF21 = 0,      /* Algorithm 2 */
@@ -180,6 +187,10 @@ ef21_status ef21_eval(ef21_ctx* ctx, double* f, double* grad_norm2, double* G);
 /* Synchronises the stream and returns the device status word: EF21_OK, or the first
  * error a kernel recorded (EF21_ERR_TIMEOUT, EF21_ERR_NONFINITE), or EF21_ERR_CUDA. */
 ef21_status ef21_poll(ef21_ctx* ctx);
+
+/* Selects the local objective (EF21_OBJECTIVE_*) used by ef21_init, ef21_step, ef21_local_grads and
+ * ef21_eval; default logistic.  Both execution paths support both objectives. */
+ef21_status ef21_set_objective(ef21_ctx* ctx, int32_t objective);
 
 /* EF21+ (Section 3.4, Algorithm 3).  With EF21_VARIANT_EF21_PLUS every step computes, per worker,
  * b_i = C(grad f_i(x)) and m_i = g_i + C(grad f_i(x) - g_i), the distortions B_i = ||b_i - grad f_i(x)||^2

@@ -70,6 +70,10 @@ class Oracle:
     def _f32(a) -> np.ndarray:
         return np.ascontiguousarray(a, dtype=np.float32)
 
+    def set_objective(self, objective: int) -> None:
+        """0: logistic loss (Eq. 19); 1: least squares (Appendix A.2).  Process-wide for this precision."""
+        self.lib.ef21o_set_objective(ctypes.c_int(objective))
+
     # -- compressor ----------------------------------------------------------
     def topk(self, v, k: int) -> Tuple[np.ndarray, np.ndarray]:
         v = self._r(v)

@@ -93,6 +93,11 @@ void ef21o_topk(const real* v, int64_t d, int64_t k, int32_t* idx, real* val) {
 /* f_i(x) = (1/m_i) sum_r log(1+exp(-y_r a_r.x)) + lam sum_j x_j^2/(1+x_j^2) */
 /* ------------------------------------------------------------------ */
 
+/* Objective used by the loss/gradient routines: 0 = logistic loss with regulariser (Section 5, Eq. 19),
+ * 1 = least squares (1/m_i) sum_r (a_r.x - y_r)^2 (Appendix A.2), same regulariser term (lam = 0 for none). */
+static int g_objective = 0;
+void ef21o_set_objective(int objective) { g_objective = objective; }
+
 static double softplus(double t) { /* log(1+exp(t)) without overflow */
     return (t > 0.0 ? t : 0.0) + log1p(exp(-fabs(t)));
 }
@@ -103,7 +108,8 @@ double ef21o_local_loss(const float* A, const float* y, int64_t m, int64_t d,
     for (int64_t r = 0; r < m; ++r) {
         double z = 0.0;
         for (int64_t j = 0; j < d; ++j) z += (double)A[r * d + j] * (double)x[j];
-        loss += softplus(-(double)y[r] * z);
+        if (g_objective == 0) loss += softplus(-(double)y[r] * z);
+        else loss += (z - (double)y[r]) * (z - (double)y[r]);
     }
     if (m > 0) loss /= (double)m;
     double reg = 0.0;
@@ -125,7 +131,8 @@ void ef21o_local_grad(const float* A, const float* y, int64_t m, int64_t d,
         double yr = (double)y[r];
         double t = yr * z;
         double rho;
-        if (t >= 0.0) { double e = exp(-t); rho = -yr * e / (1.0 + e); }
+        if (g_objective == 1) { rho = 2.0 * (z - yr); }
+        else if (t >= 0.0) { double e = exp(-t); rho = -yr * e / (1.0 + e); }
         else          { rho = -yr / (1.0 + exp(t)); }
         for (int64_t j = 0; j < d; ++j) acc[j] += rho * (double)A[r * d + j];
     }

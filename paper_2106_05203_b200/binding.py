@@ -23,6 +23,7 @@ STATUS_NAMES = {0: "EF21_OK", 1: "EF21_ERR_INVALID_ARG", 2: "EF21_ERR_STATE", 3:
 INIT_COMPRESSED, INIT_ZERO, INIT_GRADIENT = 0, 1, 2
 PATH_AUTO, PATH_LAUNCHES, PATH_PERSISTENT = 0, 1, 2
 VARIANT_EF21, VARIANT_EF21_PLUS = 0, 1
+OBJECTIVE_LOGISTIC, OBJECTIVE_LEAST_SQUARES = 0, 1
 
 # name -> (restype, argtypes); mirrors include/ef21.h
 _i32, _i64, _f32, _sz, _vp = ctypes.c_int32, ctypes.c_int64, ctypes.c_float, ctypes.c_size_t, ctypes.c_void_p
@@ -48,6 +49,7 @@ SIGNATURES = {
     "ef21_set_state": (ctypes.c_int, [_vp, _vp, _vp, _vp]),
     "ef21_eval": (ctypes.c_int, [_vp, _dp, _dp, _dp]),
     "ef21_poll": (ctypes.c_int, [_vp]),
+    "ef21_set_objective": (ctypes.c_int, [_vp, _i32]),
     "ef21_set_variant": (ctypes.c_int, [_vp, _i32]),
     "ef21_get_plus_choice": (ctypes.c_int, [_vp, _vp]),
     "ef21_set_topk_algorithm": (ctypes.c_int, [_vp, _i32]),
@@ -232,6 +234,9 @@ class EF21:
 
     def poll(self) -> int:
         return int(_lib.ef21_poll(self._h))
+
+    def set_objective(self, objective: int) -> None:
+        _check(_lib.ef21_set_objective(self._h, objective), "ef21_set_objective")
 
     def set_variant(self, variant: int) -> None:
         _check(_lib.ef21_set_variant(self._h, variant), "ef21_set_variant")

@@ -71,6 +71,13 @@ __device__ __forceinline__ float logistic_residual(float y, float z) {
     return __fdiv_rn(-y * num, 1.f + e);
 }
 
+// Residual rho_r = d loss / d margin for the two built-in objectives:
+//   objective 0: logistic loss log(1 + exp(-y z))      (Section 5, Eq. 19)
+//   objective 1: least squares (z - y)^2               (Appendix A.2)
+__device__ __forceinline__ float loss_residual(int objective, float y, float z) {
+    return objective == 0 ? logistic_residual(y, z) : 2.f * (z - y);
+}
+
 // d/dx of lambda x^2/(1+x^2) = 2 lambda x / (1+x^2)^2.
 __device__ __forceinline__ float regulariser_grad(float lambda, float x) {
     float q = fmaf(x, x, 1.f);

@@ -141,6 +141,7 @@ struct ef21_ctx {
     unsigned spin_limit;
     bool force_general_topk;
     int variant;                        // EF21_VARIANT_*
+    int objective;                      // EF21_OBJECTIVE_*
     cudaStream_t aux_stream;            // created on first use: overlaps the next threshold estimate
     cudaEvent_t ev_fork, ev_join;
     i64 launches;
@@ -251,7 +252,7 @@ ef21_status enqueue_topk_general(cudaStream_t st, const float* a, i64 pitch_a, c
 ef21_status enqueue_grads(ef21_ctx* c, bool with_loss) {
     if (c->num_tiles > 0) {
         grad_tiles_kernel<<<c->num_tiles, GRAD_BLOCK, 0, c->stream>>>(
-            c->at<float>(c->L.A), c->at<float>(c->L.y), c->x(), c->at<RowTile>(c->L.tiles), (int)c->L.ld,
+            c->at<float>(c->L.A), c->at<float>(c->L.y), c->x(), c->at<RowTile>(c->L.tiles), (int)c->L.ld, c->objective,
             c->at<float>(c->L.partial), with_loss ? c->at<double>(c->L.loss_partial) : nullptr);
         c->launches += 1;
     }
@@ -539,6 +540,7 @@ ef21_status run_persistent(ef21_ctx* c, const PersistPlan& P, int steps) {
     p.x = c->x(); p.g = c->g(); p.gi = c->gi(); p.msg_idx = c->msg_idx(); p.msg_val = c->msg_val();
     p.slots = c->at<unsigned long long>(c->L.slots); p.status = c->status();
     p.n = c->n; p.d = (int)c->d; p.ld = (int)c->L.ld; p.k = c->k; p.C = P.C; p.steps = steps;
+    p.objective = c->objective;
     p.slice_rows = 0; p.gamma = c->gamma; p.lambda = c->lambda; p.inv_n = 1.0f / (float)c->n;
     p.spin_limit = c->spin_limit; p.epoch0 = 0u;
     CU(cudaMemsetAsync(p.slots, 0, (size_t)2 * c->n * c->k * 8, c->stream));
@@ -605,6 +607,7 @@ ef21_status ef21_create(ef21_ctx** out, int32_t n, int64_t d, int32_t k, float g
     c->spin_limit = 1u << 22;
     c->force_general_topk = false;
     c->variant = EF21_VARIANT_EF21;
+    c->objective = EF21_OBJECTIVE_LOGISTIC;
     c->aux_stream = nullptr; c->ev_fork = nullptr; c->ev_join = nullptr;
     cudaError_t e = cudaMemsetAsync(c->ws + L.status, 0, 256, c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->x(), 0, (size_t)L.ld * 4, c->stream);
@@ -915,6 +918,12 @@ ef21_status ef21_get_persistent_shape(const ef21_ctx* c, int32_t* cluster_blocks
     if (cluster_blocks) *cluster_blocks = c->pk_used_cluster;
     if (rows_per_batch) *rows_per_batch = c->pk_used_rb;
     if (row_source) *row_source = c->pk_used_src;
+    return EF21_OK;
+}
+
+ef21_status ef21_set_objective(ef21_ctx* c, int32_t objective) {
+    if (!c || (objective != EF21_OBJECTIVE_LOGISTIC && objective != EF21_OBJECTIVE_LEAST_SQUARES)) return EF21_ERR_INVALID_ARG;
+    c->objective = objective;
     return EF21_OK;
 }
 

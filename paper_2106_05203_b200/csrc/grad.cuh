@@ -28,7 +28,7 @@ constexpr int GRAD_BLOCK = 256;
 // log(1+exp(-y z)) over the tile's rows.
 __global__ void __launch_bounds__(GRAD_BLOCK)
 grad_tiles_kernel(const float* __restrict__ A, const float* __restrict__ y, const float* __restrict__ x,
-                  const RowTile* __restrict__ tiles, int ld, float* __restrict__ partial,
+                  const RowTile* __restrict__ tiles, int ld, int objective, float* __restrict__ partial,
                   double* __restrict__ loss_partial) {
     __shared__ float rho[GRAD_TILE_MAX_ROWS];
     __shared__ double loss_w[GRAD_BLOCK / 32];
@@ -48,10 +48,15 @@ grad_tiles_kernel(const float* __restrict__ A, const float* __restrict__ y, cons
         z = warp_sum(z);
         if (lane == 0) {
             float yr = y[t.row0 + r];
-            rho[r] = logistic_residual(yr, z);
+            rho[r] = loss_residual(objective, yr, z);
             if (loss_partial) {
-                double u = -(double)yr * (double)z;
-                loss_acc += (u > 0.0 ? u : 0.0) + log1p(exp(-fabs(u)));
+                if (objective == 0) {
+                    double u = -(double)yr * (double)z;
+                    loss_acc += (u > 0.0 ? u : 0.0) + log1p(exp(-fabs(u)));
+                } else {
+                    double e = (double)z - (double)yr;
+                    loss_acc += e * e;
+                }
             }
         }
     }

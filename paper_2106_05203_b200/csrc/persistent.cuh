@@ -51,6 +51,7 @@ struct PersistParams {
     unsigned long long* slots; // [2][n*k]
     unsigned* status;
     int n, d, ld, k, C, steps;
+    int objective;             // 0 logistic loss, 1 least squares
     int slice_rows;            // capacity (rows) of the shared-memory slice (SMEM source)
     float gamma, lambda, inv_n;
     unsigned spin_limit;
@@ -263,7 +264,7 @@ __global__ void __launch_bounds__(THREADS, 1) persistent_kernel(const PersistPar
                     pd[r] = z;
                 }
                 const float z = reduce_rows<RB>(pd, lane);
-                const float rho = logistic_residual(y_reg, z);
+                const float rho = loss_residual(p.objective, y_reg, z);
 #pragma unroll
                 for (int r = 0; r < RB; ++r) {
                     const float pr = __shfl_sync(0xffffffffu, rho, r << SH);

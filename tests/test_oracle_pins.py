@@ -463,3 +463,54 @@ def test_ef21_plus_plain_branch_is_exercised(oracle64):
     assert st.choice.sum() == w.n
     for i in range(w.n):
         assert np.count_nonzero(st.gi[i]) <= 4
+
+
+# ---------------------------------------------------------------------------
+# Least squares objective (Appendix A.2)
+# ---------------------------------------------------------------------------
+
+@pytest.fixture
+def ls_oracle64(oracle64):
+    oracle64.set_objective(1)
+    yield oracle64
+    oracle64.set_objective(0)
+
+
+def test_least_squares_loss_and_gradient(ls_oracle64):
+    # f_i = (1/m) sum (a.x - y)^2 : closed form gradient (2/m) A^T (A x - y), and central differences
+    o = ls_oracle64
+    w = inputs.config(0)
+    rng = np.random.default_rng(8)
+    x = rng.standard_normal(w.d)
+    A = w.A[:50].astype(np.float64); y = w.y[:50].astype(np.float64)
+    res = A @ x - y
+    assert o.local_loss(w.A[:50], w.y[:50], x, 0.0) == pytest.approx(np.mean(res ** 2), rel=1e-13)
+    np.testing.assert_allclose(o.local_grad(w.A[:50], w.y[:50], x, 0.0), 2.0 * A.T @ res / 50, rtol=1e-12, atol=1e-14)
+    g = o.local_grad(w.A[:50], w.y[:50], x, 0.1)
+    h = 1e-6
+    for j in (0, 17, 63):
+        e = np.zeros(w.d); e[j] = h
+        fd = (o.local_loss(w.A[:50], w.y[:50], x + e, 0.1) - o.local_loss(w.A[:50], w.y[:50], x - e, 0.1)) / (2 * h)
+        assert fd == pytest.approx(g[j], rel=1e-6, abs=1e-8)
+
+
+def test_least_squares_ef21_converges_linearly(ls_oracle64):
+    # Theorem 2 (PL case): with the stepsize bound of Eq. 16 the Lyapunov function decreases geometrically;
+    # here only monotone decrease of f + (gamma/theta) G and a large overall drop are checked.
+    o = ls_oracle64
+    w = inputs.config(0)
+    k = 8
+    L_i = inputs.smoothness_constants(w.A, w.row_offsets, 0.0, "least_squares")
+    L, Lt = float(np.mean(L_i)), float(np.sqrt(np.mean(L_i ** 2)))
+    alpha = k / w.d
+    theta = 1 - math.sqrt(1 - alpha); beta = (1 - alpha) / (1 - math.sqrt(1 - alpha))
+    gamma = 1.0 / (L + Lt * math.sqrt(2 * beta / theta))
+    st = oracle_mod.State(o, w.n, w.d, k, gamma, 0.0, w.A, w.y, w.row_offsets, w.x0)
+    st.init(0)
+    psi = []
+    for _ in range(200):
+        _, G = o.diagnostics(w.A, w.y, w.row_offsets, st.x, 0.0, st.gi)
+        psi.append(st.loss() + gamma / theta * G)
+        st.step(1)
+    assert all(b <= a + 1e-12 for a, b in zip(psi, psi[1:]))
+    assert psi[-1] < 0.7 * psi[0]
