@@ -199,3 +199,15 @@ def config(index: int, k: Optional[int] = None, scale: float = 1.0):
         return StressWorkload("topk-stress", n=n, d=d, k=k or max(1, d // 1000), gamma=0.01,
                               T=50, seed=4)
     raise ValueError(f"no workload {index}")
+
+
+def minibatch_rows(seed: int, step: int, row_offsets: np.ndarray, tau: int) -> np.ndarray:
+    """Rows of one stochastic step: for every worker tau distinct row numbers inside its shard (sampling
+    without replacement, as in the paper's minibatch experiments), int32 [n, tau], from its own stream."""
+    rng = np.random.default_rng(np.random.PCG64([seed, 7919, step]))
+    n = len(row_offsets) - 1
+    out = np.empty((n, tau), dtype=np.int32)
+    for i in range(n):
+        m = int(row_offsets[i + 1] - row_offsets[i])
+        out[i] = rng.choice(m, size=tau, replace=False)
+    return out

@@ -197,6 +197,14 @@ class State:
         self.o.lib.ef21o_plus_round(_c_int32(self.n), _c_int64(self.d), _c_int64(self.k), _p(grads),
                                     _p(self.gi), _p(self.g), _p(self.idx), _p(self.val), _p(ch))
 
+    def step_minibatch(self, batch) -> None:
+        """One iteration of Algorithm 5 with the given rows (batch[n, tau], row numbers inside each shard)."""
+        batch = np.ascontiguousarray(batch, dtype=np.int32)
+        assert batch.shape[0] == self.n
+        self.o.lib.ef21o_step_minibatch(_c_int32(self.n), _c_int64(self.d), _c_int64(self.k), _p(self.A), _p(self.y),
+                                        _p(self.off), _c_double(self.lam), self.o._creal(self.gamma), _p(batch),
+                                        _c_int32(batch.shape[1]), *self._args_state())
+
     def round(self, grads) -> None:
         """One message round (no x update) given the local gradients."""
         grads = self.o._r(grads)

@@ -361,3 +361,30 @@ void ef21o_plus_step_grads(int32_t steps, int32_t n, int64_t d, int64_t k, const
         ef21o_plus_round(n, d, k, V, gi, g, idx, val, choice);
     }
 }
+
+/* ------------------------------------------------------------------ */
+/* Stochastic EF21 (Algorithm 5): minibatch gradient estimates          */
+/* ------------------------------------------------------------------ */
+
+/* One iteration of Algorithm 5: x <- x - gamma g; every worker forms the estimate
+ *     ghat_i = (1/tau) sum_{r in batch_i} rho_r a_r + regulariser term
+ * over the tau rows batch[i][0..tau) of its shard (row numbers inside the shard, drawn by the caller)
+ * and uses it in place of grad f_i in the message round of Algorithm 2. */
+void ef21o_step_minibatch(int32_t n, int64_t d, int64_t k, const float* A, const float* y,
+                          const int64_t* row_off, double lam, real gamma, const int32_t* batch, int32_t tau,
+                          real* x, real* gi, real* g, int32_t* idx, real* val) {
+    real* grads = (real*)malloc((size_t)n * (size_t)d * sizeof(real));
+    float* Ab = (float*)malloc((size_t)tau * (size_t)d * sizeof(float));
+    float* yb = (float*)malloc((size_t)tau * sizeof(float));
+    ef21o_x_update(d, gamma, g, x);
+    for (int32_t i = 0; i < n; ++i) {
+        for (int32_t r = 0; r < tau; ++r) {
+            const int64_t row = row_off[i] + batch[(int64_t)i * tau + r];
+            memcpy(Ab + (int64_t)r * d, A + row * d, (size_t)d * sizeof(float));
+            yb[r] = y[row];
+        }
+        ef21o_local_grad(Ab, yb, tau, d, x, lam, grads + (int64_t)i * d);
+    }
+    ef21o_round(n, d, k, grads, gi, g, idx, val);
+    free(grads); free(Ab); free(yb);
+}

@@ -514,3 +514,70 @@ def test_least_squares_ef21_converges_linearly(ls_oracle64):
         st.step(1)
     assert all(b <= a + 1e-12 for a, b in zip(psi, psi[1:]))
     assert psi[-1] < 0.7 * psi[0]
+
+
+# ---------------------------------------------------------------------------
+# Stochastic EF21 (Algorithm 5)
+# ---------------------------------------------------------------------------
+
+@pytest.mark.parametrize("precision", ["f32", "f64"])
+def test_minibatch_of_all_rows_is_the_full_step(precision):
+    # tau = m_i with the rows in their own order: Algorithm 5 is Algorithm 2
+    o = oracle_mod.Oracle(precision)
+    w = inputs.config(0)
+    m = int(np.min(np.diff(w.row_offsets)))
+    assert np.all(np.diff(w.row_offsets) == m)
+    a = oracle_mod.State(o, w.n, w.d, w.k, w.gamma, w.lam, w.A, w.y, w.row_offsets, w.x0); a.init(0)
+    b = oracle_mod.State(o, w.n, w.d, w.k, w.gamma, w.lam, w.A, w.y, w.row_offsets, w.x0); b.init(0)
+    batch = np.tile(np.arange(m, dtype=np.int32), (w.n, 1))
+    for _ in range(5):
+        a.step(1); b.step_minibatch(batch)
+        for u, v in ((a.x, b.x), (a.g, b.g), (a.gi, b.gi), (a.val, b.val)):
+            np.testing.assert_array_equal(u, v)
+        np.testing.assert_array_equal(a.idx, b.idx)
+
+
+def test_minibatch_estimate_is_the_gradient_of_the_selected_rows(oracle64):
+    # From g_i = 0 and g = 0 with k = d the first message is the whole estimate, so g_i = ghat_i; it must be
+    # the gradient of the sub-shard made of exactly the chosen rows (in particular: the right worker's rows)
+    o = oracle64
+    w = inputs.config(0)
+    tau = 7
+    batch = inputs.minibatch_rows(3, 0, w.row_offsets, tau)
+    st = oracle_mod.State(o, w.n, w.d, w.d, w.gamma, w.lam, w.A, w.y, w.row_offsets, w.x0); st.init(1)
+    st.step_minibatch(batch)
+    np.testing.assert_array_equal(st.x, w.x0.astype(np.float64))
+    for i in range(w.n):
+        rows = w.row_offsets[i] + batch[i].astype(np.int64)
+        expect = o.local_grad(w.A[rows], w.y[rows], w.x0.astype(np.float64), w.lam)
+        np.testing.assert_array_equal(st.gi[i], expect)
+    np.testing.assert_allclose(st.g, st.gi.mean(axis=0), rtol=1e-13, atol=1e-16)
+
+
+def test_minibatch_estimate_is_unbiased_over_all_subsets(oracle64):
+    # Assumption of Algorithm 5's analysis: E[ghat_i] = grad f_i.  Brute force over all C(6,3) batches.
+    import itertools
+    o = oracle64
+    rng = np.random.default_rng(21)
+    m, d, tau, lam = 6, 5, 3, 0.1
+    A = rng.standard_normal((m, d)).astype(np.float32)
+    y = np.sign(rng.standard_normal(m)).astype(np.float32)
+    x = rng.standard_normal(d)
+    off = np.array([0, m], dtype=np.int64)
+    acc = np.zeros(d); count = 0
+    for rows in itertools.combinations(range(m), tau):
+        st = oracle_mod.State(o, 1, d, d, 0.0, lam, A, y, off, x); st.init(1)
+        st.step_minibatch(np.array([rows], dtype=np.int32))
+        acc += st.gi[0]; count += 1
+    assert count == 20
+    np.testing.assert_allclose(acc / count, o.local_grad(A, y, x, lam), rtol=1e-12, atol=1e-14)
+
+
+def test_minibatch_order_only_changes_rounding(oracle64):
+    o = oracle64
+    w = inputs.config(0)
+    batch = inputs.minibatch_rows(4, 1, w.row_offsets, 16)
+    a = oracle_mod.State(o, w.n, w.d, w.d, w.gamma, w.lam, w.A, w.y, w.row_offsets, w.x0); a.init(1)
+    b = oracle_mod.State(o, w.n, w.d, w.d, w.gamma, w.lam, w.A, w.y, w.row_offsets, w.x0); b.init(1)
+    a.step_minibatch(batch); b.step_minibatch(batch[:, ::-1].copy())
+    np.testing.assert_allclose(a.gi, b.gi, rtol=1e-12, atol=1e-15)
