@@ -135,6 +135,14 @@ ef21_status ef21_step(ef21_ctx* ctx, int32_t steps);
  * passed this call. */
 ef21_status ef21_step_grads(ef21_ctx* ctx, const float* V_dev, int32_t steps);
 
+/* One iteration of the stochastic variant (Appendix, Algorithm 5): the loop of Algorithm 2 with
+ * grad f_i(x^{t+1}) replaced by the minibatch estimate over the tau rows batch_dev[i][0..tau) of worker i's
+ * shard (row numbers inside the shard, int32, leading dimension tau; the caller draws them, e.g. without
+ * replacement), averaged over tau, plus the regulariser term.  Every shard needs at least tau rows.  An
+ * index outside its shard is replaced by row 0 and EF21_ERR_INVALID_ARG is recorded in the status word
+ * (ef21_poll).  Launch path; EF21_VARIANT_EF21 only. */
+ef21_status ef21_step_minibatch(ef21_ctx* ctx, const int32_t* batch_dev, int32_t tau);
+
 /* grad f_i(x) for the current x and all workers, written to grads_out_dev[n][d]
  * (Eq. 19 differentiated; state is not changed). */
 ef21_status ef21_local_grads(ef21_ctx* ctx, float* grads_out_dev);

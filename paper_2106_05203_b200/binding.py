@@ -40,6 +40,7 @@ SIGNATURES = {
     "ef21_init_grads": (ctypes.c_int, [_vp, _vp, _i32]),
     "ef21_step": (ctypes.c_int, [_vp, _i32]),
     "ef21_step_grads": (ctypes.c_int, [_vp, _vp, _i32]),
+    "ef21_step_minibatch": (ctypes.c_int, [_vp, _vp, _i32]),
     "ef21_local_grads": (ctypes.c_int, [_vp, _vp]),
     "ef21_topk_workspace_bytes": (_sz, [_i32, _i64, _i32]),
     "ef21_topk": (ctypes.c_int, [_vp, _i32, _i64, _i32, _vp, _vp, _vp, _sz, _vp]),
@@ -191,6 +192,14 @@ class EF21:
 
     def step_grads(self, V: torch.Tensor, steps: int = 1) -> None:
         _check(_lib.ef21_step_grads(self._h, _ptr(_dev_f32(V, (self.n, self.d))), steps), "ef21_step_grads")
+
+    def step_minibatch(self, batch: torch.Tensor) -> None:
+        """One stochastic iteration; batch[n, tau] int32 row numbers inside each worker's shard."""
+        if not (batch.is_cuda and batch.dtype == torch.int32 and batch.is_contiguous() and batch.dim() == 2
+                and batch.shape[0] == self.n):
+            raise TypeError("batch must be a contiguous int32 CUDA tensor of shape [n, tau]")
+        _check(_lib.ef21_step_minibatch(self._h, _ptr(batch), int(batch.shape[1])), "ef21_step_minibatch")
+        self._keep_batch = batch
 
     def local_grads(self) -> torch.Tensor:
         out = torch.empty((self.n, self.d), dtype=torch.float32, device=self.device)

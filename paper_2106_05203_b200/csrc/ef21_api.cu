@@ -77,7 +77,7 @@ struct Layout {
     i64 max_tiles;     // capacity of the gradient tile table
     size_t status, x, g, gi, msg_idx, msg_val, topk, agg_off, eval_out, slots;
     size_t msg2_idx, msg2_val, plus_old, plus_choice, plus_bitmap;    // EF21+ (Algorithm 3)
-    size_t A, y, row_off, tile_begin, tiles, partial, loss_partial, grad;
+    size_t A, y, row_off, tile_begin, tiles, partial, loss_partial, grad, mb_tile_begin, mb_tiles;
     size_t total;
     TopkLayout tk;
 };
@@ -105,7 +105,7 @@ Layout make_layout(i64 n, i64 d, i64 k, i64 N) {
     L.plus_choice = take((size_t)n * 4);
     L.plus_bitmap = take((size_t)n * ((d + 31) / 32) * 4);
     L.tile_rows = 0; L.max_tiles = 0;
-    L.A = L.y = L.row_off = L.tile_begin = L.tiles = L.partial = L.loss_partial = L.grad = 0;
+    L.A = L.y = L.row_off = L.tile_begin = L.tiles = L.partial = L.loss_partial = L.grad = L.mb_tile_begin = L.mb_tiles = 0;
     if (N > 0) {
         L.tile_rows = grad_tile_rows(N, L.ld);
         L.max_tiles = N / L.tile_rows + n;
@@ -117,6 +117,8 @@ Layout make_layout(i64 n, i64 d, i64 k, i64 N) {
         L.partial = take((size_t)L.max_tiles * L.ld * 4);
         L.loss_partial = take((size_t)L.max_tiles * 8);
         L.grad = take((size_t)n * L.ld * 4);
+        L.mb_tile_begin = take((size_t)(n + 1) * 4);
+        L.mb_tiles = take((size_t)L.max_tiles * sizeof(RowTile));
     }
     L.total = o;
     return L;
@@ -148,6 +150,9 @@ struct ef21_ctx {
     std::vector<i64> row_off;
     std::vector<RowTile> tiles;
     std::vector<int> tile_begin;
+    std::vector<RowTile> mb_tiles;      // tile table of the minibatch lists, rebuilt when tau changes
+    std::vector<int> mb_tile_begin;
+    int mb_tau;
 
     template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
     float* x() const { return at<float>(L.x); }
@@ -253,14 +258,49 @@ ef21_status enqueue_grads(ef21_ctx* c, bool with_loss) {
     if (c->num_tiles > 0) {
         grad_tiles_kernel<<<c->num_tiles, GRAD_BLOCK, 0, c->stream>>>(
             c->at<float>(c->L.A), c->at<float>(c->L.y), c->x(), c->at<RowTile>(c->L.tiles), (int)c->L.ld, c->objective,
-            c->at<float>(c->L.partial), with_loss ? c->at<double>(c->L.loss_partial) : nullptr);
+            c->at<float>(c->L.partial), with_loss ? c->at<double>(c->L.loss_partial) : nullptr, nullptr, 0,
+            c->at<i64>(c->L.row_off), c->status());
         c->launches += 1;
     }
     dim3 grid((unsigned)ceil_div(c->L.ld, 256), (unsigned)c->n);
     grad_finish_kernel<<<grid, 256, 0, c->stream>>>(c->at<float>(c->L.partial), c->at<int>(c->L.tile_begin),
                                                     c->at<i64>(c->L.row_off), c->x(), c->lambda, (int)c->d,
-                                                    (int)c->L.ld, c->at<float>(c->L.grad));
+                                                    (int)c->L.ld, c->at<float>(c->L.grad), 0);
     c->launches += 1;
+    CU(cudaGetLastError());
+    return EF21_OK;
+}
+
+// Minibatch gradients (Algorithm 5): worker i averages over the tau rows batch[i][0..tau) of its shard.
+ef21_status enqueue_minibatch_grads(ef21_ctx* c, const int* batch_dev, int tau) {
+    if (c->mb_tau != tau) {            // (re)build the tile table of the batch lists
+        const int R = c->L.tile_rows;
+        c->mb_tiles.clear();
+        c->mb_tile_begin.assign(c->n + 1, 0);
+        for (int i = 0; i < c->n; ++i) {
+            c->mb_tile_begin[i] = (int)c->mb_tiles.size();
+            for (int r = 0; r < tau; r += R) {
+                RowTile t; t.row0 = r; t.rows = std::min(R, tau - r); t.worker = i;
+                c->mb_tiles.push_back(t);
+            }
+        }
+        c->mb_tile_begin[c->n] = (int)c->mb_tiles.size();
+        if ((i64)c->mb_tiles.size() > c->L.max_tiles) return EF21_ERR_WORKSPACE;
+        CU(cudaMemcpyAsync(c->at<int>(c->L.mb_tile_begin), c->mb_tile_begin.data(), (size_t)(c->n + 1) * 4,
+                           cudaMemcpyHostToDevice, c->stream));
+        CU(cudaMemcpyAsync(c->at<RowTile>(c->L.mb_tiles), c->mb_tiles.data(), c->mb_tiles.size() * sizeof(RowTile),
+                           cudaMemcpyHostToDevice, c->stream));
+        CU(cudaStreamSynchronize(c->stream));      // the host vectors may be rebuilt by the next call
+        c->mb_tau = tau;
+    }
+    grad_tiles_kernel<<<(unsigned)c->mb_tiles.size(), GRAD_BLOCK, 0, c->stream>>>(
+        c->at<float>(c->L.A), c->at<float>(c->L.y), c->x(), c->at<RowTile>(c->L.mb_tiles), (int)c->L.ld, c->objective,
+        c->at<float>(c->L.partial), nullptr, batch_dev, tau, c->at<i64>(c->L.row_off), c->status());
+    dim3 grid((unsigned)ceil_div(c->L.ld, 256), (unsigned)c->n);
+    grad_finish_kernel<<<grid, 256, 0, c->stream>>>(c->at<float>(c->L.partial), c->at<int>(c->L.mb_tile_begin),
+                                                    c->at<i64>(c->L.row_off), c->x(), c->lambda, (int)c->d,
+                                                    (int)c->L.ld, c->at<float>(c->L.grad), tau);
+    c->launches += 2;
     CU(cudaGetLastError());
     return EF21_OK;
 }
@@ -607,6 +647,7 @@ ef21_status ef21_create(ef21_ctx** out, int32_t n, int64_t d, int32_t k, float g
     c->spin_limit = 1u << 22;
     c->force_general_topk = false;
     c->variant = EF21_VARIANT_EF21;
+    c->mb_tau = -1;
     c->objective = EF21_OBJECTIVE_LOGISTIC;
     c->aux_stream = nullptr; c->ev_fork = nullptr; c->ev_join = nullptr;
     cudaError_t e = cudaMemsetAsync(c->ws + L.status, 0, 256, c->stream);
@@ -747,6 +788,19 @@ ef21_status ef21_step_grads(ef21_ctx* c, const float* V_dev, int32_t steps) {
         EF(enqueue_round_aggregate(c, true));
         if (sampled) CU(cudaStreamWaitEvent(c->stream, c->ev_join, 0));
     }
+    c->last_path = EF21_PATH_LAUNCHES;
+    return EF21_OK;
+}
+
+ef21_status ef21_step_minibatch(ef21_ctx* c, const int32_t* batch_dev, int32_t tau) {
+    if (!c || !batch_dev || tau < 1) return EF21_ERR_INVALID_ARG;
+    if (!c->shards_loaded || !c->inited) return EF21_ERR_STATE;
+    if (c->variant != EF21_VARIANT_EF21) return EF21_ERR_UNSUPPORTED;
+    for (int i = 0; i < c->n; ++i)
+        if (c->row_off[i + 1] - c->row_off[i] < tau) return EF21_ERR_INVALID_ARG;
+    EF(enqueue_x_update(c));
+    EF(enqueue_minibatch_grads(c, batch_dev, tau));
+    EF(enqueue_round(c, c->at<float>(c->L.grad), c->L.ld, false));
     c->last_path = EF21_PATH_LAUNCHES;
     return EF21_OK;
 }

@@ -24,21 +24,37 @@ constexpr int GRAD_TILE_MAX_ROWS = 256;
 constexpr int GRAD_BLOCK = 256;
 
 // A: [N][ld] (ld % 4 == 0, padding columns are zero), x: [ld] (padding zero).
-// partial: [num_tiles][ld].  loss_partial (optional): [num_tiles] doubles, sum of
-// log(1+exp(-y z)) over the tile's rows.
+// partial: [num_tiles][ld].  loss_partial (optional): [num_tiles] doubles, sum of the per-row losses
+// over the tile's rows.
+// gather (optional): minibatch mode.  A tile then covers positions [row0, row0 + rows) of its worker's
+// index list gather[worker * gather_pitch + ...]; each entry is a row number inside the worker's shard.
+// An entry outside the shard records EF21_ERR_INVALID_ARG in the status word and is replaced by row 0.
 __global__ void __launch_bounds__(GRAD_BLOCK)
 grad_tiles_kernel(const float* __restrict__ A, const float* __restrict__ y, const float* __restrict__ x,
                   const RowTile* __restrict__ tiles, int ld, int objective, float* __restrict__ partial,
-                  double* __restrict__ loss_partial) {
+                  double* __restrict__ loss_partial, const int* __restrict__ gather, int gather_pitch,
+                  const i64* __restrict__ row_off, unsigned* __restrict__ status) {
     __shared__ float rho[GRAD_TILE_MAX_ROWS];
+    __shared__ i64 rowid[GRAD_TILE_MAX_ROWS];
     __shared__ double loss_w[GRAD_BLOCK / 32];
     const RowTile t = tiles[blockIdx.x];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = GRAD_BLOCK / 32;
     const int chunks = ld >> 2;
+    for (int r = threadIdx.x; r < t.rows; r += GRAD_BLOCK) {
+        i64 row = t.row0 + r;
+        if (gather) {
+            const i64 lo = row_off[t.worker], m = row_off[t.worker + 1] - lo;
+            i64 pick = gather[(i64)t.worker * gather_pitch + t.row0 + r];
+            if (pick < 0 || pick >= m) { record_error(status, 1u /* EF21_ERR_INVALID_ARG */); pick = 0; }
+            row = lo + pick;
+        }
+        rowid[r] = row;
+    }
+    __syncthreads();
     const float4* __restrict__ x4 = reinterpret_cast<const float4*>(x);
     double loss_acc = 0.0;
     for (int r = warp; r < t.rows; r += nwarps) {
-        const float4* __restrict__ row = reinterpret_cast<const float4*>(A + (t.row0 + r) * (i64)ld);
+        const float4* __restrict__ row = reinterpret_cast<const float4*>(A + rowid[r] * (i64)ld);
         float z = 0.f;
         for (int c = lane; c < chunks; c += 32) {
             float4 a = row[c];
@@ -47,7 +63,7 @@ grad_tiles_kernel(const float* __restrict__ A, const float* __restrict__ y, cons
         }
         z = warp_sum(z);
         if (lane == 0) {
-            float yr = y[t.row0 + r];
+            float yr = y[rowid[r]];
             rho[r] = loss_residual(objective, yr, z);
             if (loss_partial) {
                 if (objective == 0) {
@@ -72,9 +88,8 @@ grad_tiles_kernel(const float* __restrict__ A, const float* __restrict__ y, cons
     float4* __restrict__ out = reinterpret_cast<float4*>(partial + (i64)blockIdx.x * ld);
     for (int c = threadIdx.x; c < chunks; c += GRAD_BLOCK) {
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        const float4* __restrict__ col = reinterpret_cast<const float4*>(A + t.row0 * (i64)ld) + c;
         for (int r = 0; r < t.rows; ++r) {
-            float4 a = col[(i64)r * chunks];
+            const float4 a = reinterpret_cast<const float4*>(A + rowid[r] * (i64)ld)[c];
             float p = rho[r];
             acc.x = fmaf(p, a.x, acc.x); acc.y = fmaf(p, a.y, acc.y);
             acc.z = fmaf(p, a.z, acc.z); acc.w = fmaf(p, a.w, acc.w);
@@ -87,7 +102,7 @@ grad_tiles_kernel(const float* __restrict__ A, const float* __restrict__ y, cons
 // tile_begin: [n+1] first tile of each worker; rows_of: [n] m_i.
 __global__ void grad_finish_kernel(const float* __restrict__ partial, const int* __restrict__ tile_begin,
                                    const i64* __restrict__ row_off, const float* __restrict__ x,
-                                   float lambda, int d, int ld, float* __restrict__ grad) {
+                                   float lambda, int d, int ld, float* __restrict__ grad, int batch_rows) {
     const int i = blockIdx.y;
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= ld) return;
@@ -95,7 +110,7 @@ __global__ void grad_finish_kernel(const float* __restrict__ partial, const int*
     if (j < d) {
         float acc = 0.f;
         for (int t = tile_begin[i]; t < tile_begin[i + 1]; ++t) acc = __fadd_rn(acc, partial[(i64)t * ld + j]);
-        const i64 m = row_off[i + 1] - row_off[i];
+        const i64 m = batch_rows > 0 ? (i64)batch_rows : row_off[i + 1] - row_off[i];   // minibatch: average over its rows
         float data = m > 0 ? __fdiv_rn(acc, (float)m) : 0.f;
         out = __fadd_rn(data, regulariser_grad(lambda, x[j]));
     }

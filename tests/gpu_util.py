@@ -43,21 +43,27 @@ def set_gpu_state_from_oracle(h, st):
     h.set_state(dev(st.x), dev(st.g), dev(st.gi))
 
 
-def lockstep(h, st, o, w, steps, k=None, grad_tol=1e-5):
+def lockstep(h, st, o, w, steps, k=None, grad_tol=1e-5, advance=None, grads_of=None):
     """Advance GPU and oracle one iteration at a time from a common state.
 
     Every step: the GPU's messages must equal the oracle's (indices and, up to the gradient
     tolerance, values).  Where an index differs, both choices must be valid Top-k picks of vectors
     that agree within the gradient tolerance (a near-tie); the GPU is then re-based onto the
-    oracle's state.  Returns the number of re-basings."""
+    oracle's state.  Returns the number of re-basings.
+
+    advance(t) (optional) performs iteration t on both sides instead of the plain step; grads_of(t)
+    then returns the vectors that iteration fed to the compressor (default: the full gradients)."""
     k = k or w.k
     rebased = 0
     for t in range(steps):
         gi_old = st.gi.copy()
-        h.step(1)
-        st.step(1)
+        if advance is None:
+            h.step(1)
+            st.step(1)
+        else:
+            advance(t)
         x, g, gi, li, lv = h.get_state_host()
-        grads = st.grads().astype(np.float64)
+        grads = (st.grads() if grads_of is None else grads_of(t)).astype(np.float64)
         scale = np.max(np.abs(grads), axis=1) + 1e-30
         dispute = False
         for i in range(w.n):
