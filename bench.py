@@ -116,6 +116,22 @@ def dist_env():
     return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
 
 
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """The slowest rank's time: what a whole-job throughput has to be divided by."""
+    if world == 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(units_per_rank: float, world: int, ms_max: float) -> float:
+    """Replicas only: every rank processes units_per_rank in at most ms_max milliseconds."""
+    return world * units_per_rank / (ms_max * 1e-3)
+
+
 # ---------------------------------------------------------------------------------------------
 # reference arm: the CPU oracle, as it stands, on the host cores
 # ---------------------------------------------------------------------------------------------
@@ -176,12 +192,8 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    def max_over_ranks(ms: float) -> float:
-        if world == 1:
-            return ms
-        t = torch.tensor([ms], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    def slowest(ms: float) -> float:
+        return max_over_ranks(ms, world, device)
 
     peak, peak_kind = measured_peak()
     flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=device)     # > 126 MB of L2
@@ -208,7 +220,7 @@ def run_ours(args):
         l0 = hs.launch_count
         e0.record(); hs.step_grads(V, steps); e1.record()
         barrier()
-        ms = max_over_ranks(e0.elapsed_time(e1))
+        ms = slowest(e0.elapsed_time(e1))
         b = stress_bytes_per_iteration(n_w, ws.d, ws.k)
         gbs = b * steps / (ms * 1e-3) / 1e9
         return {"workload": f"configs[4] {ws.name}: n={n_w} d={ws.d} Top-{ws.k} supplied gradients (static)",
@@ -253,7 +265,7 @@ def run_ours(args):
             e1.record()
             barrier()
             launches = h.launch_count - l0
-            times.append(max_over_ranks(e0.elapsed_time(e1)))
+            times.append(slowest(e0.elapsed_time(e1)))
         if sampler:
             # nvidia-smi cannot resolve a few milliseconds: keep the same launches running for a while
             # longer (untimed) so that the sampler sees the clocks under exactly this load
@@ -274,7 +286,7 @@ def run_ours(args):
     steps = args.steps if args.steps is not None else w.T
     warmup = max(3, args.warmup if args.warmup is not None else 20)
     r = time_logistic(w, w.k, steps, warmup, with_clocks=True)
-    its = world * steps / (r["ms"] * 1e-3)
+    its = whole_job_rate(steps, world, r["ms"])
     bytes_iter = logistic_bytes_per_iteration(w.n, w.d, w.k, w.N)
     achieved = bytes_iter * steps / (r["ms"] * 1e-3) / 1e9
     path_name = {1: "launch-per-stage kernels", 2: "persistent_kernel (one launch for all iterations)"}.get(r["path"], "?")
@@ -299,9 +311,9 @@ def run_ours(args):
         h2.init(B.INIT_COMPRESSED)
         h2.step(steps)
         xh, gh, _, _, _ = h2.get_state_host(want_gi=False, messages=False)      # synchronises
-        e2e_times.append(max_over_ranks((time.perf_counter() - t0) * 1e3))
+        e2e_times.append(slowest((time.perf_counter() - t0) * 1e3))
     e2e_ms = statistics.median(e2e_times) if e2e_times else float("nan")
-    e2e = None if args.no_e2e else {"value": world * steps / (e2e_ms * 1e-3), "unit": UNIT,
+    e2e = None if args.no_e2e else {"value": whole_job_rate(steps, world, e2e_ms), "unit": UNIT,
            "h2d_bytes_per_step": (w.A.nbytes + w.y.nbytes) / steps, "d2h_bytes_per_step": (xh.nbytes + gh.nbytes) / steps,
            "note": f"create + load_shards_host + init + {steps} iterations + get_state_host, pinned host buffers; "
                    "bytes are per run divided by the iterations of the run"}
