@@ -138,6 +138,7 @@ struct ef21_ctx {
     bool shards_loaded, inited;
     int num_tiles;
     int path, last_path;
+    bool agg_off_ready;                 // the last selection already wrote the aggregation's tile offsets
     int pk_cluster, pk_rb, pk_src, pk_threads;      // forced persistent-kernel shape (0 / -1 = automatic)
     int pk_used_cluster, pk_used_rb, pk_used_src, pk_used_threads;
     unsigned spin_limit;
@@ -216,7 +217,8 @@ ef21_status enqueue_topk_fast_sample(cudaStream_t st, const float* a, i64 pitch_
 // is given, g_i += c_i is applied by the same kernel that writes the messages.
 ef21_status enqueue_topk_fast(cudaStream_t st, const float* a, i64 pitch_a, const float* b, i64 pitch_b,
                               int batch, i64 d, int k, int* idx_out, float* val_out, float* gi_rows, i64 ld,
-                              const TopkBuffers& B, i64* launches, bool sampled = false) {
+                              const TopkBuffers& B, i64* launches, bool sampled = false, int* tile_off = nullptr,
+                              int ntiles = 0) {
     static bool smem_set = false;
     const size_t finish_smem = (size_t)ST_CAND_CAP * 12 + 2048 * 4;
     if (!smem_set) {
@@ -229,7 +231,8 @@ ef21_status enqueue_topk_fast(cudaStream_t st, const float* a, i64 pitch_a, cons
     auto collect = vec ? st_collect_kernel<true> : st_collect_kernel<false>;
     collect<<<grid, ST_COLLECT_WARPS * 32, 0, st>>>(a, pitch_a, b, pitch_b, d, B.nreg, B.thr, B.cand, B.region_cnt, B.flags);
     st_finish_kernel<<<batch, ST_THREADS, finish_smem, st>>>(a, pitch_a, b, pitch_b, d, B.nreg, k, B.cand, B.region_cnt,
-                                                             B.flags, idx_out, val_out, gi_rows, ld, B.slow_count);
+                                                             B.flags, idx_out, val_out, gi_rows, ld, B.slow_count, tile_off,
+                                                             ntiles, AGG_TILE);
     if (launches) *launches += 2;
     CU(cudaGetLastError());
     return EF21_OK;
@@ -310,9 +313,12 @@ ef21_status enqueue_minibatch_grads(ef21_ctx* c, const int* batch_dev, int tau) 
 ef21_status enqueue_round_select(ef21_ctx* c, const float* a, i64 pitch_a, bool sampled) {
     TopkBuffers B = topk_buffers(c->ws + c->L.topk, c->L.tk);
     if (B.fast && !c->force_general_topk) {
+        // the finish kernel also leaves the per-tile offsets of the messages for the aggregation
         EF(enqueue_topk_fast(c->stream, a, pitch_a, c->gi(), c->L.ld, c->n, c->d, c->k, c->msg_idx(), c->msg_val(),
-                             c->gi(), c->L.ld, B, &c->launches, sampled));
+                             c->gi(), c->L.ld, B, &c->launches, sampled, c->at<int>(c->L.agg_off), c->L.agg_tiles));
+        c->agg_off_ready = true;
     } else {
+        c->agg_off_ready = false;
         EF(enqueue_topk_general(c->stream, a, pitch_a, c->gi(), c->L.ld, c->n, c->d, c->k, c->msg_idx(),
                                 c->msg_val(), B, &c->launches));
         const i64 total = (i64)c->n * c->k;
@@ -326,16 +332,20 @@ ef21_status enqueue_round_select(ef21_ctx* c, const float* a, i64 pitch_a, bool 
 
 // Aggregation half: g += (1/n) sum c_i (and, if update_x, x <- x - gamma g_old in the same kernel).
 ef21_status enqueue_round_aggregate(ef21_ctx* c, bool update_x) {
-    const i64 noff = (i64)c->n * (c->L.agg_tiles + 1);
-    agg_offsets_kernel<<<(unsigned)ceil_div(noff, 256), 256, 0, c->stream>>>(c->msg_idx(), c->n, c->k,
-                                                                            c->L.agg_tiles, c->at<int>(c->L.agg_off));
+    if (!c->agg_off_ready) {
+        const i64 noff = (i64)c->n * (c->L.agg_tiles + 1);
+        agg_offsets_kernel<<<(unsigned)ceil_div(noff, 256), 256, 0, c->stream>>>(c->msg_idx(), c->n, c->k,
+                                                                                c->L.agg_tiles, c->at<int>(c->L.agg_off));
+        c->launches += 1;
+    }
+    c->agg_off_ready = false;
     const float inv_n = 1.0f / (float)c->n;
     auto kern = c->n <= AGG_STAGE_MAX_N
                     ? (update_x ? aggregate_staged_kernel<true> : aggregate_staged_kernel<false>)
                     : (update_x ? aggregate_kernel<true> : aggregate_kernel<false>);
     kern<<<c->L.agg_tiles, AGG_BLOCK, 0, c->stream>>>(c->msg_idx(), c->msg_val(), c->at<int>(c->L.agg_off), c->n, c->k,
                                                       c->L.agg_tiles, c->d, inv_n, c->gamma, c->g(), c->x());
-    c->launches += 2;
+    c->launches += 1;
     CU(cudaGetLastError());
     return EF21_OK;
 }
@@ -642,7 +652,7 @@ ef21_status ef21_create(ef21_ctx** out, int32_t n, int64_t d, int32_t k, float g
     c->L = L;
     c->shards_loaded = false; c->inited = false; c->num_tiles = 0;
     c->path = EF21_PATH_AUTO; c->last_path = 0; c->launches = 0;
-    c->pk_cluster = 0; c->pk_rb = 0; c->pk_src = -1; c->pk_threads = 0;
+    c->pk_cluster = 0; c->pk_rb = 0; c->pk_src = -1; c->pk_threads = 0; c->agg_off_ready = false;
     c->pk_used_cluster = c->pk_used_rb = 0; c->pk_used_src = -1; c->pk_used_threads = 0;
     c->spin_limit = 1u << 22;
     c->force_general_topk = false;
@@ -764,8 +774,6 @@ ef21_status ef21_step_grads(ef21_ctx* c, const float* V_dev, int32_t steps) {
     }
     const bool fast = c->L.tk.fast && !c->force_general_topk;
     if (fast && steps > 1 && !c->aux_stream) {
-        // V is the same at every step, so the threshold estimate of step t+1 only waits for the
-        // g_i update of step t and can run beside the aggregation of step t on a second stream.
         if (cudaStreamCreateWithFlags(&c->aux_stream, cudaStreamNonBlocking) != cudaSuccess ||
             cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
             cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess) {
@@ -774,20 +782,33 @@ ef21_status ef21_step_grads(ef21_ctx* c, const float* V_dev, int32_t steps) {
         }
     }
     TopkBuffers B = topk_buffers(c->ws + c->L.topk, c->L.tk);
-    bool sampled = false;
-    for (int t = 0; t < steps; ++t) {
-        EF(enqueue_round_select(c, V_dev, c->d, sampled));
-        sampled = false;
-        if (fast && t + 1 < steps) {
-            CU(cudaEventRecord(c->ev_fork, c->stream));
-            CU(cudaStreamWaitEvent(c->aux_stream, c->ev_fork, 0));
-            EF(enqueue_topk_fast_sample(c->aux_stream, V_dev, c->d, c->gi(), c->L.ld, c->n, c->d, c->k, B, &c->launches));
-            CU(cudaEventRecord(c->ev_join, c->aux_stream));
-            sampled = true;
+    if (!(fast && steps > 1)) {
+        for (int t = 0; t < steps; ++t) {
+            EF(enqueue_round_select(c, V_dev, c->d, false));
+            EF(enqueue_round_aggregate(c, true));
         }
-        EF(enqueue_round_aggregate(c, true));
-        if (sampled) CU(cudaStreamWaitEvent(c->stream, c->ev_join, 0));
+        c->last_path = EF21_PATH_LAUNCHES;
+        return EF21_OK;
     }
+    // Same V at every step: the threshold estimate of round t+1 needs V and g_i^{t+1} only, so it
+    // follows the finish kernel of round t directly on this stream, and the aggregation of round t (g
+    // and x) runs beside it on the second stream; the streaming pass of round t+1 waits for both.
+    cudaStream_t main_stream = c->stream;
+    for (int t = 0; t < steps; ++t) {
+        // (letting the streaming pass start while the aggregation still runs made the pass 15-20 % slower)
+        if (t > 0) CU(cudaStreamWaitEvent(main_stream, c->ev_join, 0));
+        EF(enqueue_round_select(c, V_dev, c->d, t > 0));
+        CU(cudaEventRecord(c->ev_fork, main_stream));
+        CU(cudaStreamWaitEvent(c->aux_stream, c->ev_fork, 0));
+        c->stream = c->aux_stream;
+        const ef21_status agg = enqueue_round_aggregate(c, true);
+        c->stream = main_stream;
+        EF(agg);
+        CU(cudaEventRecord(c->ev_join, c->aux_stream));
+        if (t + 1 < steps)
+            EF(enqueue_topk_fast_sample(main_stream, V_dev, c->d, c->gi(), c->L.ld, c->n, c->d, c->k, B, &c->launches));
+    }
+    CU(cudaStreamWaitEvent(main_stream, c->ev_join, 0));
     c->last_path = EF21_PATH_LAUNCHES;
     return EF21_OK;
 }

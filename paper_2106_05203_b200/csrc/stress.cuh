@@ -11,7 +11,9 @@
 //   3. finish:   one block per vector stages the candidates in shared memory, finds the exact k-th
 //                key by radix select, breaks ties toward the lower index by an ordered scan, writes
 //                the k pairs in ascending index order and stores g_i + c_i on the selected
-//                coordinates (no read-modify-write: the new value came with the candidate).
+//                coordinates (no read-modify-write: the new value came with the candidate).  On
+//                request it also writes where each tile of coordinates begins in the message (the
+//                offsets the aggregation needs), so no separate search kernel runs.
 // The threshold only decides speed, never the result: if a vector ends up with fewer than k
 // candidates, more than the staging capacity, or an overflowing region, its finish block runs the
 // exact selection over the whole vector instead (slow, same output bit for bit).
@@ -243,7 +245,8 @@ __global__ void __launch_bounds__(ST_THREADS, 1)
 st_finish_kernel(const float* a, i64 pitch_a, const float* b, i64 pitch_b, i64 d, int nreg, int k,
                  const int4* __restrict__ cand, const int* __restrict__ region_cnt,
                  const unsigned* __restrict__ flags, int* __restrict__ idx_out, float* __restrict__ val_out,
-                 float* gi_rows, i64 ld, unsigned* __restrict__ slow_count) {
+                 float* gi_rows, i64 ld, unsigned* __restrict__ slow_count,
+                 int* __restrict__ tile_off, int ntiles, int tile) {
     extern __shared__ __align__(16) unsigned char st_smem[];
     __shared__ unsigned scratch[33];
     __shared__ unsigned res[3];
@@ -258,8 +261,10 @@ st_finish_kernel(const float* a, i64 pitch_a, const float* b, i64 pitch_b, i64 d
     float* __restrict__ vo = val_out + (i64)i * k;
     float* gi_row = gi_rows ? gi_rows + (i64)i * ld : nullptr;
 
-    // stage the candidates in index order: per group of 1024 regions, prefix-sum the region counts,
-    // then copy with one thread per candidate (its region found by binary search in the prefix)
+    // stage the candidates in index order: per group of 1024 regions, prefix-sum the region counts
+    // (thread t holds region r0 + t), then every warp copies the lists of its 32 regions, eight
+    // regions in flight, one lane per candidate
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     unsigned total = 0u;
     bool bad = flags[i] != 0u;
     for (int r0 = 0; r0 < nreg; r0 += ST_THREADS) {
@@ -267,30 +272,30 @@ st_finish_kernel(const float* a, i64 pitch_a, const float* b, i64 pitch_b, i64 d
         const unsigned c = r < nreg ? (unsigned)region_cnt[(i64)i * nreg + r] : 0u;
         unsigned tot;
         const unsigned pre = block_excl_scan(c, scratch, tot);
-        hist[threadIdx.x] = pre;                      // hist doubles as the prefix array here
-        __syncthreads();
         if (!bad && total + tot <= (unsigned)ST_CAND_CAP) {
-            constexpr int U = 8;                         // candidates in flight per thread
-            for (unsigned eb = 0; eb < tot; eb += U * ST_THREADS) {
+            const int4* __restrict__ src = cand + ((i64)i * nreg + r0 + warp * 32) * ST_REGION_CAP;
+            constexpr int U = 8;
+            for (int rr0 = 0; rr0 < 32; rr0 += U) {
                 int4 w[U];
+                unsigned cu[U], pu[U];
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
-                    const unsigned e = eb + u * ST_THREADS + threadIdx.x;
-                    if (e < tot) {
-                        int lo = 0, hi = ST_THREADS;     // last region with prefix <= e
-                        while (hi - lo > 1) {
-                            const int mid = (lo + hi) >> 1;
-                            if (hist[mid] <= e) lo = mid; else hi = mid;
-                        }
-                        w[u] = cand[((i64)i * nreg + r0 + lo) * ST_REGION_CAP + (e - hist[lo])];
-                    }
+                    cu[u] = __shfl_sync(0xffffffffu, c, rr0 + u);
+                    pu[u] = __shfl_sync(0xffffffffu, pre, rr0 + u);
+                    if ((unsigned)lane < cu[u]) w[u] = src[(rr0 + u) * ST_REGION_CAP + lane];
                 }
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
-                    const unsigned e = eb + u * ST_THREADS + threadIdx.x;
-                    if (e < tot) {
-                        cidx[total + e] = w[u].x; cval[total + e] = __int_as_float(w[u].y);
-                        cnew[total + e] = __int_as_float(w[u].z);
+                    if ((unsigned)lane < cu[u]) {
+                        const unsigned at = total + pu[u] + (unsigned)lane;
+                        cidx[at] = w[u].x; cval[at] = __int_as_float(w[u].y); cnew[at] = __int_as_float(w[u].z);
+                    }
+                    for (unsigned more = 32u; more < cu[u]; more += 32u) {       // rare: a list longer than a warp
+                        if (more + (unsigned)lane < cu[u]) {
+                            const int4 x = src[(rr0 + u) * ST_REGION_CAP + more + lane];
+                            const unsigned at = total + pu[u] + more + (unsigned)lane;
+                            cidx[at] = x.x; cval[at] = __int_as_float(x.y); cnew[at] = __int_as_float(x.z);
+                        }
                     }
                 }
             }
@@ -301,6 +306,19 @@ st_finish_kernel(const float* a, i64 pitch_a, const float* b, i64 pitch_b, i64 d
     if (bad || total < (unsigned)k || total > (unsigned)ST_CAND_CAP) {
         if (threadIdx.x == 0 && slow_count) atomicAdd(slow_count, 1u);
         st_slow_exact(av, bv, d, k, io, vo, gi_row, hist, scratch, res);
+        if (tile_off) {
+            __syncthreads();                         // the block's own writes to io are visible to it now
+            int* off = tile_off + (i64)i * (ntiles + 1);
+            for (int b = threadIdx.x; b <= ntiles; b += ST_THREADS) {
+                const i64 bound = (i64)b * tile;
+                int lo = 0, hi = k;
+                while (lo < hi) {
+                    const int mid = (lo + hi) >> 1;
+                    if ((i64)io[mid] < bound) lo = mid + 1; else hi = mid;
+                }
+                off[b] = lo;
+            }
+        }
         return;
     }
 
@@ -328,22 +346,41 @@ st_finish_kernel(const float* a, i64 pitch_a, const float* b, i64 pitch_b, i64 d
     }
     unsigned tot;
     const unsigned packed = block_excl_scan(n_ge | (n_tie << 16), scratch, tot);
-    unsigned my_ge = packed & 0xffffu, my_tie = packed >> 16;
-    for (unsigned e = e0; e < e1; ++e) {
-        const float val = cval[e];
-        const unsigned key = mag_key(val);
-        const bool is_ge = key >= s.lo_ge;
-        const bool is_tie = s.need_ties && key == s.T;
-        if (is_ge || (is_tie && my_tie < s.need_ties)) {
-            const unsigned pos = is_ge ? my_ge + min(my_tie, s.need_ties) : my_ge + my_tie;
-            if (pos < (unsigned)k) {
-                const int j = cidx[e];
-                io[pos] = j; vo[pos] = val;
-                if (gi_row) gi_row[j] = cnew[e];           // g_i + c_i, computed when the entry was read
+    // Pass A: the state update g_i + c_i on the selected coordinates (scattered stores).  Pass B, after
+    // everybody has read its cnew entries: the selected (index, value) pairs go, compacted and in
+    // order, into the space of cnew.  Pass C writes them out with coalesced stores and derives, from
+    // neighbouring indices, where each tile of `tile` coordinates starts in the message.
+    int2* out2 = reinterpret_cast<int2*>(cnew);                 // [k] <= ST_CAND_CAP / 2 pairs
+    for (int pass = 0; pass < 2; ++pass) {
+        unsigned my_ge = packed & 0xffffu, my_tie = packed >> 16;
+        for (unsigned e = e0; e < e1; ++e) {
+            const float val = cval[e];
+            const unsigned key = mag_key(val);
+            const bool is_ge = key >= s.lo_ge;
+            const bool is_tie = s.need_ties && key == s.T;
+            if (is_ge || (is_tie && my_tie < s.need_ties)) {
+                const unsigned pos = is_ge ? my_ge + min(my_tie, s.need_ties) : my_ge + my_tie;
+                if (pos < (unsigned)k) {
+                    if (pass == 0) { if (gi_row) gi_row[cidx[e]] = cnew[e]; }      // g_i + c_i, computed when the entry was read
+                    else out2[pos] = make_int2(cidx[e], __float_as_int(val));
+                }
             }
+            my_ge += is_ge ? 1u : 0u;
+            my_tie += is_tie ? 1u : 0u;
         }
-        my_ge += is_ge ? 1u : 0u;
-        my_tie += is_tie ? 1u : 0u;
+        __syncthreads();
+    }
+    int* off = tile_off ? tile_off + (i64)i * (ntiles + 1) : nullptr;
+    for (int p0 = threadIdx.x; p0 < k; p0 += ST_THREADS) {
+        const int2 me = out2[p0];
+        io[p0] = me.x; vo[p0] = __int_as_float(me.y);
+        if (off) {
+            const int t_prev = p0 > 0 ? out2[p0 - 1].x / tile : -1;
+            const int t_me = me.x / tile;
+            for (int b = t_prev + 1; b <= t_me; ++b) off[b] = p0;          // tiles that begin at this entry
+            if (p0 == k - 1)
+                for (int b = t_me + 1; b <= ntiles; ++b) off[b] = k;       // nothing left for the tiles behind the last entry
+        }
     }
 }
 
