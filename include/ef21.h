@@ -132,7 +132,9 @@ ef21_status ef21_step(ef21_ctx* ctx, int32_t steps);
 /* The same loop with grad f_i replaced by the caller's V_dev[n][d], re-used unchanged at
  * each of the `steps` iterations (the static input sequence of Section 3.1); call with
  * steps = 1 and fresh V for a changing sequence.  V must stay valid until the stream has
- * passed this call. */
+ * passed this call.  With steps > 1 on long vectors the library orders part of the work on a second
+ * stream of its own (created on first use, joined back into the handle's stream before the call's
+ * work ends), so a later operation on the handle's stream still sees the complete result. */
 ef21_status ef21_step_grads(ef21_ctx* ctx, const float* V_dev, int32_t steps);
 
 /* One iteration of the stochastic variant (Appendix, Algorithm 5): the loop of Algorithm 2 with
