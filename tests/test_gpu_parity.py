@@ -217,6 +217,21 @@ def test_free_running_tiny_T100(path, B, oracle32):
     assert h.poll() == 0
 
 
+@pytest.mark.parametrize("cfg", [1, 2])
+def test_free_running_paper_shapes_full_T(cfg, B, oracle32):
+    """The benchmark's own runs: workloads [1] and [2] (Top-1), T = 2,000 iterations in the launch configuration
+    that bench.py times (automatic path and shape), against 2,000 oracle iterations: x and f(x) within 1e-4."""
+    w = inputs.config(cfg)
+    h = make_gpu(w); st = make_oracle_state(oracle32, w)
+    h.init(0); st.init(0)
+    h.step(w.T); st.step(w.T)
+    assert w.T == 2000 and h.last_path == B.PATH_PERSISTENT
+    x = h.get_state_host()[0]
+    assert rel_l2(x, st.x) <= 1e-4
+    assert h.eval()[0] == pytest.approx(st.loss(), rel=1e-4)
+    assert h.poll() == 0
+
+
 @PATHS
 @pytest.mark.parametrize("cfg,k,steps", [(1, 1, 150), (2, 1, 40), (2, 4, 40), (2, 16, 40), (3, 1, 25)])
 def test_lockstep_paper_shapes(cfg, k, steps, path, B, oracle32):
