@@ -18,7 +18,8 @@ rank, _, world = bench.dist_env()
 dist.init_process_group("gloo")
 ms = bench.max_over_ranks(10.0 + 5.0 * rank, world, "cpu")
 rate = bench.whole_job_rate(2000, world, ms)
-print(json.dumps({"rank": rank, "world": world, "ms": ms, "rate": rate}), flush=True)
+# one os.write per rank: two ranks' lines never share a line of the merged output
+os.write(1, (json.dumps({"rank": rank, "world": world, "ms": ms, "rate": rate}) + "\n").encode())
 dist.destroy_process_group()
 """
 
