@@ -487,8 +487,13 @@ struct PersistPlan {
     PersistKernel kernel;
 };
 
-size_t pk_smem_bytes(int ld, int C, int nmsg, int src, i64 rows_cta, int threads) {
+// From two entries per worker on, the received messages are scattered into a [n][ld] table in shared
+// memory (if that table is small): aggregation then costs n reads per coordinate instead of n*k.
+bool pk_use_table(int n, int ld, int k) { return k >= 2 && (size_t)n * ld * 4 <= (size_t)PK_TABLE_MAX_BYTES; }
+
+size_t pk_smem_bytes(int n, int k, int ld, int C, int nmsg, int src, i64 rows_cta, int threads) {
     size_t b = (size_t)(6 + threads / 32 + C) * ld * 4 + (size_t)((nmsg + 1) & ~1) * 8 + (size_t)((2 * ld + 15) & ~15);
+    if (pk_use_table(n, ld, k)) b += (size_t)n * ld * 4;
     if (src == PK_SRC_SMEM) b += (size_t)rows_cta * ld * 4;
     return b;
 }
@@ -521,7 +526,7 @@ PersistPlan plan_persistent(ef21_ctx* c) {
             if (ceil_div(rows_cta, cand) <= 16) { rb = cand; src = PK_SRC_REG; threads = 512; }
         if (!rb) {
             rb = max_rb512; threads = 512;
-            src = pk_smem_bytes(ld, C, nmsg, PK_SRC_SMEM, rows_cta, threads) <= (size_t)max_smem - 1024 ? PK_SRC_SMEM : PK_SRC_GMEM;
+            src = pk_smem_bytes(c->n, c->k, ld, C, nmsg, PK_SRC_SMEM, rows_cta, threads) <= (size_t)max_smem - 1024 ? PK_SRC_SMEM : PK_SRC_GMEM;
         }
         if (c->pk_threads > 0) {
             threads = c->pk_threads;
@@ -561,7 +566,7 @@ PersistPlan plan_persistent(ef21_ctx* c) {
         const i64 rows_cta = shape_for(C, rb, src, threads);
         if (c->pk_cluster == 0 && C > 1 && rows_cta < 8) continue;       // do not split below one batch
         if (src == PK_SRC_REG && ceil_div(rows_cta, rb) > threads / 32) continue;
-        const size_t smem = pk_smem_bytes(ld, C, nmsg, src, rows_cta, threads);
+        const size_t smem = pk_smem_bytes(c->n, c->k, ld, C, nmsg, src, rows_cta, threads);
         if (smem > (size_t)max_smem - 1024) continue;
         PersistKernel kern = pk_lookup(chunk_slots, rb, src, threads);
         if (!kern) continue;
@@ -591,7 +596,7 @@ ef21_status run_persistent(ef21_ctx* c, const PersistPlan& P, int steps) {
     p.slots = c->at<unsigned long long>(c->L.slots); p.status = c->status();
     p.n = c->n; p.d = (int)c->d; p.ld = (int)c->L.ld; p.k = c->k; p.C = P.C; p.steps = steps;
     p.objective = c->objective;
-    p.slice_rows = 0; p.gamma = c->gamma; p.lambda = c->lambda; p.inv_n = 1.0f / (float)c->n;
+    p.slice_rows = 0; p.use_table = pk_use_table(c->n, (int)c->L.ld, c->k) ? 1 : 0; p.gamma = c->gamma; p.lambda = c->lambda; p.inv_n = 1.0f / (float)c->n;
     p.spin_limit = c->spin_limit; p.epoch0 = 0u;
     CU(cudaMemsetAsync(p.slots, 0, (size_t)2 * c->n * c->k * 8, c->stream));
     cudaLaunchConfig_t cfg = {};

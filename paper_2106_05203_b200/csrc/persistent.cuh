@@ -37,6 +37,8 @@ constexpr int PK_MAX_THREADS = 512;     // the kernel is instantiated for 256 an
 constexpr int PK_MAX_K = 32;
 constexpr int PK_MAX_MSGS = 2048;       // n*k words staged in shared memory
 constexpr int PK_SCAN_MAX_MSGS = 128;   // up to this many messages every coordinate thread scans them all
+constexpr int PK_TABLE_MAX_BYTES = 64 * 1024;   // largest [n][ld] message table kept in shared memory
+constexpr unsigned PK_NO_ENTRY = 0xffffffffu;   // table cell without a message (a NaN pattern no finite value has)
 enum { PK_SRC_REG = 0, PK_SRC_SMEM = 1, PK_SRC_GMEM = 2 };
 
 struct PersistParams {
@@ -53,6 +55,7 @@ struct PersistParams {
     int n, d, ld, k, C, steps;
     int objective;             // 0 logistic loss, 1 least squares
     int slice_rows;            // capacity (rows) of the shared-memory slice (SMEM source)
+    int use_table;             // 1: received messages are scattered into a [n][ld] table in shared memory
     float gamma, lambda, inv_n;
     unsigned spin_limit;
     unsigned epoch0;           // epoch of the first iteration minus one
@@ -163,7 +166,8 @@ __global__ void __launch_bounds__(THREADS, 1) persistent_kernel(const PersistPar
     float* sacc = reinterpret_cast<float*>(msg + ((nmsg + 1) & ~1));                  // [ld] per-coordinate sum of messages
     unsigned char* touched = reinterpret_cast<unsigned char*>(sacc + ld);             // [ld] coordinate received a message
     unsigned char* sel = touched + ld;                                                // [ld] leader: entry is in the Top-k
-    float* slice = reinterpret_cast<float*>(touched + ((2 * ld + 15) & ~15));         // SMEM source, 16-byte aligned
+    unsigned* table = reinterpret_cast<unsigned*>(touched + ((2 * ld + 15) & ~15));   // [n][ld] value bits by (worker, coordinate)
+    float* slice = reinterpret_cast<float*>(table + (p.use_table ? p.n * ld : 0));    // SMEM source, 16-byte aligned
     __shared__ int abort_flag;
     __shared__ __align__(8) unsigned long long part_bar;     // leader: counts the bytes of the partials
 
@@ -187,6 +191,8 @@ __global__ void __launch_bounds__(THREADS, 1) persistent_kernel(const PersistPar
     }
     for (int j = tid; j < ld; j += THREADS) { xs[j] = p.x[j]; gs[j] = p.g[j]; }
     for (int j = tid; j < ld; j += THREADS) { sacc[j] = 0.f; touched[j] = 0; }
+    if (p.use_table)
+        for (int e = tid; e < p.n * ld; e += THREADS) table[e] = PK_NO_ENTRY;
     if (SRC == PK_SRC_SMEM) {
         const float4* src = reinterpret_cast<const float4*>(p.A + r0 * (i64)ld);
         float4* dst = reinterpret_cast<float4*>(slice);
@@ -232,6 +238,7 @@ __global__ void __launch_bounds__(THREADS, 1) persistent_kernel(const PersistPar
 #pragma unroll
         for (int e = 0; e < 4; ++e)
             if (4 * (lane + 32 * cs) + e >= p.d) pad_mask |= 1u << (cs * 4 + e);
+    const unsigned k_magic = (65536u + (unsigned)p.k - 1u) / (unsigned)p.k;     // u / k == (u * k_magic) >> 16 for u < 2048, k <= 32
     bool aborted = false;
     for (int t = 0; t < p.steps; ++t) {
         const unsigned epoch = (p.epoch0 + (unsigned)t + 1u) & 0xffffu;
@@ -427,17 +434,42 @@ __global__ void __launch_bounds__(THREADS, 1) persistent_kernel(const PersistPar
             for (int u = tid; u < nmsg; u += THREADS) {
                 unsigned spins = 0;
                 unsigned long long w;
+                bool got = true;
                 while (true) {
                     w = ld_relaxed_u64(slot + u);
                     if ((unsigned)(w >> 48) == epoch) break;
                     ++spins;
-                    if ((spins & 1023u) == 0u && ld_relaxed_u32(p.status) != 0u) { abort_flag = 1; break; }
-                    if (spins > p.spin_limit) { record_error(p.status, (unsigned)5 /* EF21_ERR_TIMEOUT */); abort_flag = 1; break; }
+                    if ((spins & 1023u) == 0u && ld_relaxed_u32(p.status) != 0u) { abort_flag = 1; got = false; break; }
+                    if (spins > p.spin_limit) { record_error(p.status, (unsigned)5 /* EF21_ERR_TIMEOUT */); abort_flag = 1; got = false; break; }
                 }
-                msg[u] = w;
+                if (p.use_table) {
+                    const unsigned idx = (unsigned)(w >> 32) & 0xffffu;
+                    if (got && idx < (unsigned)ld) table[(int)(((unsigned)u * k_magic) >> 16) * ld + (int)idx] = (unsigned)w;
+                } else {
+                    msg[u] = w;
+                }
             }
             __syncthreads();
             if (abort_flag) aborted = true;
+        }
+        if (!aborted && p.use_table) {
+            // g_j += (1/n) * sum over workers (ascending) of the values sent for coordinate j: row i of the
+            // table holds worker i's message scattered by coordinate; a cell is emptied by the thread that
+            // read it (the next messages are written several barriers later)
+            for (int j = tid; j < p.d; j += THREADS) {
+                float s = 0.f; bool hit = false;
+#pragma unroll 4
+                for (int i = 0; i < p.n; ++i) {
+                    const unsigned bits = table[i * ld + j];
+                    const bool present = bits != PK_NO_ENTRY;
+                    const float sum = __fadd_rn(s, __uint_as_float(bits));
+                    s = present ? sum : s;
+                    hit = hit || present;
+                    table[i * ld + j] = PK_NO_ENTRY;
+                }
+                if (hit) gs[j] = __fadd_rn(gs[j], __fmul_rn(s, p.inv_n));
+            }
+            continue;
         }
         if (!aborted && nmsg > PK_SCAN_MAX_MSGS) {
             // many messages: warp 0 folds them into per-coordinate running sums, one worker at a time (a
