@@ -219,3 +219,50 @@ class State:
 
     def grads(self) -> np.ndarray:
         return self.o.all_grads(self.A, self.y, self.off, self.x, self.lam)
+
+
+class EFState:
+    """State of the original error feedback method (Algorithm 4) on the oracle: x, the errors e_i, the
+    stepsize-scaled gradients a_i = gamma * grad f_i(x) at the current x and the messages w_i last sent."""
+
+    def __init__(self, oracle: Oracle, n: int, d: int, k: int, gamma: float, lam: float = 0.0,
+                 A=None, y=None, row_offsets=None, x0=None):
+        self.o = oracle
+        self.n, self.d, self.k = int(n), int(d), int(k)
+        self.gamma = float(gamma)
+        self.lam = float(lam)
+        self.A = None if A is None else Oracle._f32(A)
+        self.y = None if y is None else Oracle._f32(y)
+        self.off = None if row_offsets is None else np.ascontiguousarray(row_offsets, dtype=np.int64)
+        real = oracle.real
+        self.x = np.zeros(d, dtype=real) if x0 is None else np.array(x0, dtype=real)
+        self.e = np.zeros((n, d), dtype=real)
+        self.a = np.zeros((n, d), dtype=real)
+        self.idx = np.zeros((n, k), dtype=np.int32)
+        self.val = np.zeros((n, k), dtype=real)
+
+    def _state(self):
+        return (_p(self.x), _p(self.e), _p(self.a), _p(self.idx), _p(self.val))
+
+    def init(self) -> None:
+        self.o.lib.ef21o_ef_init(_c_int32(self.n), _c_int64(self.d), _c_int64(self.k), _p(self.A), _p(self.y),
+                                 _p(self.off), _c_double(self.lam), self.o._creal(self.gamma), *self._state())
+
+    def init_from_grads(self, grads) -> None:
+        grads = self.o._r(grads)
+        self.o.lib.ef21o_ef_init_from_grads(_c_int32(self.n), _c_int64(self.d), _c_int64(self.k),
+                                            self.o._creal(self.gamma), _p(grads), *self._state()[1:])
+
+    def step(self, steps: int = 1) -> None:
+        self.o.lib.ef21o_ef_step(_c_int32(steps), _c_int32(self.n), _c_int64(self.d), _c_int64(self.k),
+                                 _p(self.A), _p(self.y), _p(self.off), _c_double(self.lam),
+                                 self.o._creal(self.gamma), *self._state())
+
+    def step_grads(self, V, steps: int = 1) -> None:
+        V = self.o._r(V)
+        assert V.shape == (self.n, self.d)
+        self.o.lib.ef21o_ef_step_grads(_c_int32(steps), _c_int32(self.n), _c_int64(self.d), _c_int64(self.k),
+                                       _p(V), self.o._creal(self.gamma), *self._state())
+
+    def loss(self) -> float:
+        return self.o.loss(self.A, self.y, self.off, self.x, self.lam)

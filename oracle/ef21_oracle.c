@@ -29,8 +29,12 @@
  * Parity pins: see tests/test_oracle_*.py (finite differences, closed forms,
  * brute-force sort, k = d => gradient descent, n = 1 => Algorithm 1, the
  * contraction bound of Eq. 3, the one-step distortion bound from the proof of
- * Lemma 2, Theorem 1, a hand-worked Algorithm 2 example).  The stepsize rule
- * gamma = 1/L is a harness convention: parity unpinned by the paper.
+ * Lemma 2, Theorem 1, a hand-worked Algorithm 2 example).  The original error
+ * feedback method (Algorithm 4) at the end of the file is pinned by a
+ * hand-worked run, the perturbed-iterate identity x - mean e, the contraction
+ * of the error, Theorem 3 for the identity compressor and an exact check of
+ * every rounding.  The stepsize rule gamma = 1/L is a harness convention:
+ * parity unpinned by the paper.
  */
 #include <math.h>
 #include <stdint.h>
@@ -387,4 +391,109 @@ void ef21o_step_minibatch(int32_t n, int64_t d, int64_t k, const float* A, const
     }
     ef21o_round(n, d, k, grads, gi, g, idx, val);
     free(grads); free(Ab); free(yb);
+}
+
+/* ------------------------------------------------------------------ */
+/* EF, the original error feedback method (Algorithm 4)                */
+/* ------------------------------------------------------------------ */
+
+/* State of Algorithm 4 between iterations: x, the errors e_i, the messages w_i last sent (idx/val,
+ * k pairs per worker) and a_i = gamma * grad f_i(x) at the current x (the vector each worker
+ * "would like" to send; it is needed again by the error update of the next iteration).
+ * Each of  gamma * grad,  e + a,  (e + a) - w,  s * (1/n),  x - p  is one rounded operation. */
+
+/* Messages of one round: w_i = C(e_i + a_i) for every worker. */
+static void ef_messages(int32_t n, int64_t d, int64_t k, const real* e, const real* a, int32_t* idx, real* val) {
+    real* p = (real*)malloc((size_t)d * sizeof(real));
+    for (int32_t i = 0; i < n; ++i) {
+        for (int64_t j = 0; j < d; ++j) p[j] = e[(int64_t)i * d + j] + a[(int64_t)i * d + j];
+        ef21o_topk(p, d, k, idx + (int64_t)i * k, val + (int64_t)i * k);
+    }
+    free(p);
+}
+
+static void ef_scale(int32_t n, int64_t d, real gamma, const real* grads, real* a) {
+    for (int64_t e = 0; e < (int64_t)n * d; ++e) a[e] = gamma * grads[e];
+}
+
+/* Algorithm 4, the two lines before the loop, given the local gradients at x^0:
+ *     e_i^0 = 0,   w_i^0 = C(gamma grad f_i(x^0)). */
+void ef21o_ef_init_from_grads(int32_t n, int64_t d, int64_t k, real gamma, const real* grads,
+                              real* e, real* a, int32_t* idx, real* val) {
+    memset(e, 0, (size_t)n * (size_t)d * sizeof(real));
+    ef_scale(n, d, gamma, grads, a);
+    ef_messages(n, d, k, e, a, idx, val);
+}
+
+/* Algorithm 4, the part of one loop iteration that precedes the new gradient:
+ *     master:  x^{t+1} = x^t - (1/n) sum_i w_i^t      (per coordinate: sum over ascending i from 0,
+ *                                                      one multiply by 1/n, one subtraction)
+ *     nodes:   e_i^{t+1} = e_i^t + gamma grad f_i(x^t) - w_i^t */
+static void ef_master_and_error(int32_t n, int64_t d, int64_t k, const int32_t* idx, const real* val,
+                                const real* a, real* x, real* e) {
+    real* s = (real*)calloc((size_t)d, sizeof(real));
+    unsigned char* touched = (unsigned char*)calloc((size_t)d, 1);
+    for (int32_t i = 0; i < n; ++i)
+        for (int64_t t = 0; t < k; ++t) {
+            const int64_t j = idx[(int64_t)i * k + t];
+            s[j] = s[j] + val[(int64_t)i * k + t];
+            touched[j] = 1;
+        }
+    const real inv_n = (real)1 / (real)n;
+    for (int64_t j = 0; j < d; ++j)
+        if (touched[j]) {
+            const real p = s[j] * inv_n;
+            x[j] = x[j] - p;
+        }
+    free(s); free(touched);
+    real* w = (real*)malloc((size_t)d * sizeof(real));
+    for (int32_t i = 0; i < n; ++i) {
+        for (int64_t j = 0; j < d; ++j) w[j] = 0;
+        for (int64_t t = 0; t < k; ++t) w[idx[(int64_t)i * k + t]] = val[(int64_t)i * k + t];
+        real* ei = e + (int64_t)i * d;
+        const real* ai = a + (int64_t)i * d;
+        for (int64_t j = 0; j < d; ++j) {
+            const real want = ei[j] + ai[j];
+            ei[j] = want - w[j];
+        }
+    }
+    free(w);
+}
+
+/* One whole iteration of Algorithm 4's loop given the local gradients at the NEW point
+ * (callers that supply gradients pass them in; grads_new is grad f_i(x^{t+1})):
+ *     a_i <- gamma grad f_i(x^{t+1}),   w_i^{t+1} = C(e_i^{t+1} + a_i). */
+static void ef_new_messages(int32_t n, int64_t d, int64_t k, real gamma, const real* grads_new,
+                            const real* e, real* a, int32_t* idx, real* val) {
+    ef_scale(n, d, gamma, grads_new, a);
+    ef_messages(n, d, k, e, a, idx, val);
+}
+
+void ef21o_ef_init(int32_t n, int64_t d, int64_t k, const float* A, const float* y, const int64_t* row_off,
+                   double lam, real gamma, const real* x, real* e, real* a, int32_t* idx, real* val) {
+    real* grads = (real*)malloc((size_t)n * (size_t)d * sizeof(real));
+    ef21o_all_grads(n, d, A, y, row_off, x, lam, grads);
+    ef21o_ef_init_from_grads(n, d, k, gamma, grads, e, a, idx, val);
+    free(grads);
+}
+
+void ef21o_ef_step(int32_t steps, int32_t n, int64_t d, int64_t k, const float* A, const float* y,
+                   const int64_t* row_off, double lam, real gamma,
+                   real* x, real* e, real* a, int32_t* idx, real* val) {
+    real* grads = (real*)malloc((size_t)n * (size_t)d * sizeof(real));
+    for (int32_t t = 0; t < steps; ++t) {
+        ef_master_and_error(n, d, k, idx, val, a, x, e);
+        ef21o_all_grads(n, d, A, y, row_off, x, lam, grads);
+        ef_new_messages(n, d, k, gamma, grads, e, a, idx, val);
+    }
+    free(grads);
+}
+
+/* The same loop with caller-supplied gradients V[n][d] standing in for grad f_i at every point. */
+void ef21o_ef_step_grads(int32_t steps, int32_t n, int64_t d, int64_t k, const real* V, real gamma,
+                         real* x, real* e, real* a, int32_t* idx, real* val) {
+    for (int32_t t = 0; t < steps; ++t) {
+        ef_master_and_error(n, d, k, idx, val, a, x, e);
+        ef_new_messages(n, d, k, gamma, V, e, a, idx, val);
+    }
 }

@@ -581,3 +581,122 @@ def test_minibatch_order_only_changes_rounding(oracle64):
     b = oracle_mod.State(o, w.n, w.d, w.d, w.gamma, w.lam, w.A, w.y, w.row_offsets, w.x0); b.init(1)
     a.step_minibatch(batch); b.step_minibatch(batch[:, ::-1].copy())
     np.testing.assert_allclose(a.gi, b.gi, rtol=1e-12, atol=1e-15)
+
+
+# ---------------------------------------------------------------------------------------------
+# EF, the original error feedback method (Algorithm 4)
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("precision", ["f32", "f64"])
+def test_alg4_hand_worked_example(precision):
+    o = oracle_mod.Oracle(precision)
+    kv = _read_kv(os.path.join(GOLDEN, "alg4_hand_example.txt"))
+    V = np.array([kv["grad1"], kv["grad2"]])
+    st = oracle_mod.EFState(o, 2, 3, 1, kv["gamma"][0])
+    st.init_from_grads(V)
+    np.testing.assert_array_equal(st.x, 0.0)
+    np.testing.assert_array_equal(st.e, 0.0)
+    np.testing.assert_array_equal(st.idx[:, 0], kv["idx0"])
+    np.testing.assert_array_equal(st.val[:, 0], kv["val0"])
+    for t in (1, 2, 3):
+        st.step_grads(V, 1)
+        np.testing.assert_array_equal(st.x, kv[f"x{t}"])
+        np.testing.assert_array_equal(st.e, [kv[f"e1_{t}"], kv[f"e2_{t}"]])
+        np.testing.assert_array_equal(st.idx[:, 0], kv[f"idx{t}"])
+        np.testing.assert_array_equal(st.val[:, 0], kv[f"val{t}"])
+
+
+def test_alg4_perturbed_iterate_follows_gradient_descent(oracle64):
+    # Summing Algorithm 4's error update over the nodes and adding the master line gives, for
+    # xt^t = x^t - (1/n) sum_i e_i^t, the exact recursion xt^{t+1} = xt^t - gamma grad f(x^t):
+    # whatever the compressor dropped stays in the errors.  The identity fails for a wrong sign, a
+    # dropped term or a wrong worker/coordinate index anywhere in the loop.
+    w = inputs.config(0)
+    gamma = 0.05
+    st = oracle_mod.EFState(oracle64, w.n, w.d, w.k, gamma, w.lam, w.A, w.y, w.row_offsets, w.x0)
+    st.init()
+    for _ in range(30):
+        x_old, e_old = st.x.copy(), st.e.copy()
+        grad_old = oracle64.all_grads(w.A, w.y, w.row_offsets, x_old, w.lam).mean(axis=0)
+        idx_old, val_old = st.idx.copy(), st.val.copy()
+        st.step(1)
+        lhs = st.x - st.e.mean(axis=0)
+        rhs = x_old - e_old.mean(axis=0) - gamma * grad_old
+        np.testing.assert_allclose(lhs, rhs, rtol=0, atol=1e-14)
+        # master line: x moves by the mean of the messages that were in flight
+        wsum = np.zeros(w.d)
+        for i in range(w.n):
+            wsum[idx_old[i]] += val_old[i]
+        np.testing.assert_allclose(st.x, x_old - wsum / w.n, rtol=0, atol=1e-15)
+        # the new messages are Top-k of e^{t+1} + gamma grad f_i(x^{t+1}), and nothing else is sent
+        grads_new = oracle64.all_grads(w.A, w.y, w.row_offsets, st.x, w.lam)
+        for i in range(w.n):
+            ib, vb = _brute_topk(st.e[i] + gamma * grads_new[i], w.k)
+            np.testing.assert_array_equal(st.idx[i], ib)
+            np.testing.assert_allclose(st.val[i], vb, rtol=0, atol=1e-15)
+
+
+def test_alg4_error_is_what_the_compressor_dropped(oracle64):
+    # e_i^{t+1} = (e_i^t + gamma grad f_i(x^t)) - C(e_i^t + gamma grad f_i(x^t)): zero exactly on the k kept
+    # coordinates, and by Eq. 3 its squared norm is at most (1 - k/d) times that of the compressed vector.
+    w = inputs.config(0)
+    gamma = 0.05
+    st = oracle_mod.EFState(oracle64, w.n, w.d, w.k, gamma, w.lam, w.A, w.y, w.row_offsets, w.x0)
+    st.init()
+    for _ in range(10):
+        want = st.e + gamma * oracle64.all_grads(w.A, w.y, w.row_offsets, st.x, w.lam)
+        idx = st.idx.copy()
+        st.step(1)
+        for i in range(w.n):
+            assert np.all(st.e[i][idx[i]] == 0.0)
+            rest = np.setdiff1d(np.arange(w.d), idx[i])
+            np.testing.assert_allclose(st.e[i][rest], want[i][rest], rtol=0, atol=1e-16)
+            assert np.sum(st.e[i] ** 2) <= (1 - w.k / w.d) * np.sum(want[i] ** 2) * (1 + 1e-12)
+
+
+def test_alg4_equals_alg2_for_the_identity_compressor(oracle64):
+    # Theorem 3: for a deterministic, positively homogeneous and additive compressor EF and EF21 produce
+    # the same iterates.  Top-k with k = d is the identity, which is all three; both methods are then
+    # gradient descent (Section 5.2) and the errors stay zero.
+    w = inputs.config(0)
+    gamma = 0.1
+    ef = oracle_mod.EFState(oracle64, w.n, w.d, w.d, gamma, w.lam, w.A, w.y, w.row_offsets, w.x0)
+    ef.init()
+    st = oracle_mod.State(oracle64, w.n, w.d, w.d, gamma, w.lam, w.A, w.y, w.row_offsets, w.x0)
+    st.init(0)
+    x_gd = np.array(w.x0, dtype=np.float64)
+    for _ in range(25):
+        x_gd = x_gd - gamma * oracle64.all_grads(w.A, w.y, w.row_offsets, x_gd, w.lam).mean(axis=0)
+        ef.step(1)
+        st.step(1)
+        np.testing.assert_allclose(ef.x, st.x, rtol=0, atol=1e-13)
+        np.testing.assert_allclose(ef.x, x_gd, rtol=0, atol=1e-13)
+        np.testing.assert_allclose(ef.e, 0.0, rtol=0, atol=1e-16)
+
+
+def test_alg4_fp32_updates_are_single_rounded_operations(oracle32):
+    # every update of the fp32 state is one IEEE operation: gamma*grad, e + a, (e + a) - w, s/n, x - p
+    rng = np.random.default_rng(5)
+    n, d, k = 3, 40, 5
+    V = rng.standard_normal((n, d)).astype(np.float32)
+    gamma = np.float32(0.3)
+    st = oracle_mod.EFState(oracle32, n, d, k, float(gamma))
+    st.init_from_grads(V)
+    a = gamma * V
+    np.testing.assert_array_equal(st.a, a)
+    e = np.zeros((n, d), dtype=np.float32)
+    x = np.zeros(d, dtype=np.float32)
+    for _ in range(6):
+        idx, val = st.idx.copy(), st.val.copy()
+        st.step_grads(V, 1)
+        s = np.zeros(d, dtype=np.float32); hit = np.zeros(d, dtype=bool)
+        for i in range(n):
+            for t in range(k):
+                s[idx[i, t]] = np.float32(s[idx[i, t]] + val[i, t]); hit[idx[i, t]] = True
+        p = (s * np.float32(np.float32(1) / np.float32(n))).astype(np.float32)
+        x = np.where(hit, (x - p).astype(np.float32), x)
+        for i in range(n):
+            wv = np.zeros(d, dtype=np.float32); wv[idx[i]] = val[i]
+            e[i] = ((e[i] + a[i]).astype(np.float32) - wv).astype(np.float32)
+        np.testing.assert_array_equal(st.x.view(np.uint32), x.view(np.uint32))
+        np.testing.assert_array_equal(st.e.view(np.uint32), e.view(np.uint32))
