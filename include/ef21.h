@@ -85,7 +85,8 @@ enum {
 /* Which method ef21_step / ef21_step_grads run. */
 enum {
     EF21_VARIANT_EF21 = 0,      /* Algorithm 2 */
-    EF21_VARIANT_EF21_PLUS = 1  /* Algorithm 3: per worker the better of C and the Markov compressor */
+    EF21_VARIANT_EF21_PLUS = 1, /* Algorithm 3: per worker the better of C and the Markov compressor */
+    EF21_VARIANT_EF = 2         /* Algorithm 4: the original error feedback method (Section 4.1) */
 };
 
 const char* ef21_status_string(ef21_status s);
@@ -209,6 +210,18 @@ ef21_status ef21_set_objective(ef21_ctx* ctx, int32_t objective);
  * the launch path only (EF21_PATH_PERSISTENT returns EF21_ERR_UNSUPPORTED).  The "last message" of
  * ef21_get_state is the compressed vector that was used.  Initialisation is that of Algorithm 2. */
 ef21_status ef21_set_variant(ef21_ctx* ctx, int32_t variant);
+/* The original error feedback method, EF (Section 4.1, Algorithm 4), with EF21_VARIANT_EF.  The
+ * per-worker state is the error e_i, kept where Algorithm 2 keeps g_i (the gi argument of
+ * ef21_get_state / ef21_set_state); g is not used.  Algorithm 4 starts from e_i^0 = 0: call
+ * ef21_init(ctx, EF21_INIT_ZERO).  One step from (x^t, e_i^t) computes
+ *     w_i^t = C(e_i^t + gamma grad f_i(x^t)),   x^{t+1} = x^t - (1/n) sum_i w_i^t,
+ *     e_i^{t+1} = e_i^t + gamma grad f_i(x^t) - w_i^t
+ * so after t steps the state is Algorithm 4's (x^t, e_i^t); the algorithm's own loop forms w_i^{t+1}
+ * at the end of iteration t, here it is formed at the start of the next step from the same x^{t+1}
+ * and e_i^{t+1}.  The "last message" of ef21_get_state is w_i^{t-1}.  gamma * grad, the sum with
+ * e_i, the difference with w_i, the factor 1/n and the update of x are single rounded fp32
+ * operations; the sum over workers runs in ascending worker order.  ef21_step_grads uses the
+ * supplied vectors in place of grad f_i.  Launch path only; ef21_step_minibatch is not available. */
 /* choice_host[n]: 0 where the last EF21+ step kept the Markov compressor, 1 where it took C(grad);
  * synchronises. */
 ef21_status ef21_get_plus_choice(ef21_ctx* ctx, int32_t* choice_host);

@@ -22,7 +22,7 @@ STATUS_NAMES = {0: "EF21_OK", 1: "EF21_ERR_INVALID_ARG", 2: "EF21_ERR_STATE", 3:
                 4: "EF21_ERR_CUDA", 5: "EF21_ERR_TIMEOUT", 6: "EF21_ERR_NONFINITE", 7: "EF21_ERR_UNSUPPORTED"}
 INIT_COMPRESSED, INIT_ZERO, INIT_GRADIENT = 0, 1, 2
 PATH_AUTO, PATH_LAUNCHES, PATH_PERSISTENT = 0, 1, 2
-VARIANT_EF21, VARIANT_EF21_PLUS = 0, 1
+VARIANT_EF21, VARIANT_EF21_PLUS, VARIANT_EF = 0, 1, 2
 OBJECTIVE_LOGISTIC, OBJECTIVE_LEAST_SQUARES = 0, 1
 
 # name -> (restype, argtypes); mirrors include/ef21.h

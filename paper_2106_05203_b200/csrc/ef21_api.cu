@@ -10,6 +10,7 @@
 
 #include "apply.cuh"
 #include "common.cuh"
+#include "ef.cuh"
 #include "grad.cuh"
 #include "persistent.cuh"
 #include "plus.cuh"
@@ -330,8 +331,15 @@ ef21_status enqueue_round_select(ef21_ctx* c, const float* a, i64 pitch_a, bool 
     return EF21_OK;
 }
 
+ef21_status enqueue_aggregate_into(ef21_ctx* c, float* target, float factor, bool update_x);
+
 // Aggregation half: g += (1/n) sum c_i (and, if update_x, x <- x - gamma g_old in the same kernel).
 ef21_status enqueue_round_aggregate(ef21_ctx* c, bool update_x) {
+    return enqueue_aggregate_into(c, c->g(), 1.0f / (float)c->n, update_x);
+}
+
+// target_j += factor * (sum over workers, ascending, of the values sent for coordinate j).
+ef21_status enqueue_aggregate_into(ef21_ctx* c, float* target, float factor, bool update_x) {
     if (!c->agg_off_ready) {
         const i64 noff = (i64)c->n * (c->L.agg_tiles + 1);
         agg_offsets_kernel<<<(unsigned)ceil_div(noff, 256), 256, 0, c->stream>>>(c->msg_idx(), c->n, c->k,
@@ -339,12 +347,11 @@ ef21_status enqueue_round_aggregate(ef21_ctx* c, bool update_x) {
         c->launches += 1;
     }
     c->agg_off_ready = false;
-    const float inv_n = 1.0f / (float)c->n;
     auto kern = c->n <= AGG_STAGE_MAX_N
                     ? (update_x ? aggregate_staged_kernel<true> : aggregate_staged_kernel<false>)
                     : (update_x ? aggregate_kernel<true> : aggregate_kernel<false>);
     kern<<<c->L.agg_tiles, AGG_BLOCK, 0, c->stream>>>(c->msg_idx(), c->msg_val(), c->at<int>(c->L.agg_off), c->n, c->k,
-                                                      c->L.agg_tiles, c->d, inv_n, c->gamma, c->g(), c->x());
+                                                      c->L.agg_tiles, c->d, factor, c->gamma, target, c->x());
     c->launches += 1;
     CU(cudaGetLastError());
     return EF21_OK;
@@ -378,6 +385,30 @@ ef21_status enqueue_plus_round(ef21_ctx* c, const float* a, i64 pitch_a) {
     c->launches += 2;
     CU(cudaGetLastError());
     return EF21_OK;
+}
+
+// One iteration of the original error feedback method (Algorithm 4) on local gradients a, from the
+// state (x, e_i): e_i becomes p_i = e_i + gamma a_i, the messages are w_i = C(p_i), the master moves
+// x by -(1/n) sum w_i, and e_i <- p_i - w_i.
+ef21_status enqueue_ef_round(ef21_ctx* c, const float* a, i64 pitch_a) {
+    TopkBuffers B = topk_buffers(c->ws + c->L.topk, c->L.tk);
+    const unsigned blocks = (unsigned)std::min<i64>(ceil_div((i64)c->n * c->d, 256), 148 * 16);
+    ef_compose_kernel<<<blocks, 256, 0, c->stream>>>(a, pitch_a, c->gi(), c->L.ld, c->n, c->d, c->gamma);
+    c->launches += 1;
+    if (B.fast && !c->force_general_topk) {
+        EF(enqueue_topk_fast(c->stream, c->gi(), c->L.ld, nullptr, 0, c->n, c->d, c->k, c->msg_idx(), c->msg_val(),
+                             nullptr, 0, B, &c->launches));
+    } else {
+        EF(enqueue_topk_general(c->stream, c->gi(), c->L.ld, nullptr, 0, c->n, c->d, c->k, c->msg_idx(), c->msg_val(), B,
+                                &c->launches));
+    }
+    const i64 total = (i64)c->n * c->k;
+    ef_subtract_sent_kernel<<<(unsigned)ceil_div(total, 256), 256, 0, c->stream>>>(c->msg_idx(), c->msg_val(), total, c->k,
+                                                                                  c->L.ld, c->gi());
+    c->launches += 1;
+    c->agg_off_ready = false;
+    CU(cudaGetLastError());
+    return enqueue_aggregate_into(c, c->x(), -(1.0f / (float)c->n), false);
 }
 
 ef21_status enqueue_x_update(ef21_ctx* c) {
@@ -738,6 +769,15 @@ ef21_status ef21_step(ef21_ctx* c, int32_t steps) {
     if (!c || steps < 0) return EF21_ERR_INVALID_ARG;
     if (!c->shards_loaded || !c->inited) return EF21_ERR_STATE;
     if (steps == 0) return EF21_OK;
+    if (c->variant == EF21_VARIANT_EF) {
+        if (c->path == EF21_PATH_PERSISTENT) return EF21_ERR_UNSUPPORTED;
+        for (int t = 0; t < steps; ++t) {
+            EF(enqueue_grads(c, false));
+            EF(enqueue_ef_round(c, c->at<float>(c->L.grad), c->L.ld));
+        }
+        c->last_path = EF21_PATH_LAUNCHES;
+        return EF21_OK;
+    }
     if (c->variant == EF21_VARIANT_EF21_PLUS) {
         if (c->path == EF21_PATH_PERSISTENT) return EF21_ERR_UNSUPPORTED;
         for (int t = 0; t < steps; ++t) {
@@ -769,6 +809,11 @@ ef21_status ef21_step(ef21_ctx* c, int32_t steps) {
 ef21_status ef21_step_grads(ef21_ctx* c, const float* V_dev, int32_t steps) {
     if (!c || !V_dev || steps < 0) return EF21_ERR_INVALID_ARG;
     if (!c->inited) return EF21_ERR_STATE;
+    if (c->variant == EF21_VARIANT_EF) {
+        for (int t = 0; t < steps; ++t) EF(enqueue_ef_round(c, V_dev, c->d));
+        c->last_path = EF21_PATH_LAUNCHES;
+        return EF21_OK;
+    }
     if (c->variant == EF21_VARIANT_EF21_PLUS) {
         for (int t = 0; t < steps; ++t) {
             EF(enqueue_x_update(c));
@@ -1008,7 +1053,7 @@ ef21_status ef21_set_objective(ef21_ctx* c, int32_t objective) {
 }
 
 ef21_status ef21_set_variant(ef21_ctx* c, int32_t variant) {
-    if (!c || (variant != EF21_VARIANT_EF21 && variant != EF21_VARIANT_EF21_PLUS)) return EF21_ERR_INVALID_ARG;
+    if (!c || variant < EF21_VARIANT_EF21 || variant > EF21_VARIANT_EF) return EF21_ERR_INVALID_ARG;
     c->variant = variant;
     return EF21_OK;
 }
