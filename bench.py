@@ -35,7 +35,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (read + write) of one persistent_kernel launch of 2,000 iterations on the headline workload,
 # from the ncu capture summarised in profiles/persistent_kernel__headline_n20_d112.md.  Reported only for
 # that launch size; None otherwise.
-HEADLINE_TRAFFIC = {"steps": 2000, "bytes": 3746048}
+HEADLINE_TRAFFIC = {"steps": 2000, "bytes": 3749632}
 
 
 def logistic_bytes_per_iteration(n, d, k, N):

@@ -487,7 +487,11 @@ PersistKernel pk_by_src(int src) {
 
 // Instantiated shapes: (chunk slots per lane, rows per warp batch, threads per block).  512 threads
 // leave 128 registers per thread, so they exist only where a batch needs at most 16 float4 registers.
-PersistKernel pk_lookup(int chunks, int rb, int src, int threads) {
+PersistKernel pk_lookup(int chunks, int rb, int src, int threads, int extra) {
+    // batches of 16 + 1 rows: registers only, one chunk slot, 16 warps
+    if (extra == 1 && chunks == 1 && rb == 16 && src == PK_SRC_REG && threads == 512)
+        return persistent_kernel<1, 16, PK_SRC_REG, 512, 1>;
+    if (extra != 0) return nullptr;
     switch (chunks * 10000 + rb * 100 + threads / 256) {
         case 10401: return pk_by_src<1, 4, 256>(src);
         case 10801: return pk_by_src<1, 8, 256>(src);
@@ -513,7 +517,7 @@ PersistKernel pk_lookup(int chunks, int rb, int src, int threads) {
 
 struct PersistPlan {
     bool ok;
-    int C, rb, src, chunks, threads;
+    int C, rb, src, chunks, threads, extra;
     size_t smem;
     PersistKernel kernel;
 };
@@ -548,13 +552,17 @@ PersistPlan plan_persistent(ef21_ctx* c) {
 
     // One candidate shape for a cluster size: rows in registers with 8 warps if they fit, else with 16
     // warps, else staged in shared memory or streamed from L2 with 16 warps.
-    auto shape_for = [&](int C, int& rb, int& src, int& threads) {
+    auto shape_for = [&](int C, int& rb, int& src, int& threads, int& extra) {
         const i64 rows_cta = ceil_div(std::max<i64>(max_m, 1), C);
-        rb = 0;
+        rb = 0; extra = 0;
         for (int cand = 8; cand <= max_rb256 && !rb; cand *= 2)
             if (ceil_div(rows_cta, cand) <= 8) { rb = cand; src = PK_SRC_REG; threads = 256; }
         for (int cand = 4; cand <= max_rb512 && !rb; cand *= 2)
             if (ceil_div(rows_cta, cand) <= 16) { rb = cand; src = PK_SRC_REG; threads = 512; }
+        // one row more than 16 per warp still fits the registers of 16 warps (one chunk slot)
+        if (!rb && chunk_slots == 1 && ceil_div(rows_cta, 17) <= 16 && c->pk_threads == 0 && c->pk_rb == 0 && c->pk_src < 0) {
+            rb = 16; extra = 1; src = PK_SRC_REG; threads = 512;
+        }
         if (!rb) {
             rb = max_rb512; threads = 512;
             src = pk_smem_bytes(c->n, c->k, ld, C, nmsg, PK_SRC_SMEM, rows_cta, threads) <= (size_t)max_smem - 1024 ? PK_SRC_SMEM : PK_SRC_GMEM;
@@ -582,8 +590,8 @@ PersistPlan plan_persistent(ef21_ctx* c) {
         int pref = 0;
         for (int C = 1; C <= 8 && !pref; ++C) {
             if ((i64)c->n * C > sms) break;
-            int rb, src, threads;
-            shape_for(C, rb, src, threads);
+            int rb, src, threads, extra;
+            shape_for(C, rb, src, threads, extra);
             if (src == PK_SRC_REG && threads == 256 && rb <= 16) pref = C;
         }
         if (pref) order[norder++] = pref;
@@ -593,13 +601,13 @@ PersistPlan plan_persistent(ef21_ctx* c) {
     for (int oi = 0; oi < norder; ++oi) {
         const int C = order[oi];
         if ((i64)c->n * C > sms) continue;
-        int rb = 0, src = PK_SRC_GMEM, threads = 256;
-        const i64 rows_cta = shape_for(C, rb, src, threads);
+        int rb = 0, src = PK_SRC_GMEM, threads = 256, extra = 0;
+        const i64 rows_cta = shape_for(C, rb, src, threads, extra);
         if (c->pk_cluster == 0 && C > 1 && rows_cta < 8) continue;       // do not split below one batch
-        if (src == PK_SRC_REG && ceil_div(rows_cta, rb) > threads / 32) continue;
+        if (src == PK_SRC_REG && ceil_div(rows_cta, rb + extra) > threads / 32) continue;
         const size_t smem = pk_smem_bytes(c->n, c->k, ld, C, nmsg, src, rows_cta, threads);
         if (smem > (size_t)max_smem - 1024) continue;
-        PersistKernel kern = pk_lookup(chunk_slots, rb, src, threads);
+        PersistKernel kern = pk_lookup(chunk_slots, rb, src, threads, extra);
         if (!kern) continue;
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
             cudaGetLastError();
@@ -614,7 +622,7 @@ PersistPlan plan_persistent(ef21_ctx* c) {
         int active = 0;
         if (cudaOccupancyMaxActiveClusters(&active, kern, &cfg) != cudaSuccess) { cudaGetLastError(); continue; }
         if (active < c->n) continue;
-        P.ok = true; P.C = C; P.rb = rb; P.src = src; P.chunks = chunk_slots; P.threads = threads; P.smem = smem; P.kernel = kern;
+        P.ok = true; P.C = C; P.rb = rb; P.src = src; P.chunks = chunk_slots; P.threads = threads; P.extra = extra; P.smem = smem; P.kernel = kern;
         return P;
     }
     return P;

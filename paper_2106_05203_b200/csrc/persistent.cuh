@@ -138,13 +138,17 @@ __device__ __forceinline__ float comp_of(const float4& v, int c) {
     return c == 0 ? v.x : (c == 1 ? v.y : (c == 2 ? v.z : v.w));
 }
 
-template <int CHUNKS, int RB, int SRC, int THREADS>
+// EXTRA > 0: a warp's batch has RB + EXTRA rows; the first RB go through the transposed reduction, each
+// extra row through a plain butterfly sum (for shards whose rows per warp just exceed a power of two).
+template <int CHUNKS, int RB, int SRC, int THREADS, int EXTRA = 0>
 __global__ void __launch_bounds__(THREADS, 1) persistent_kernel(const PersistParams p) {
+    constexpr int RBT = RB + EXTRA;                                            // rows per batch
     constexpr int SH = (RB == 32) ? 0 : (RB == 16 ? 1 : (RB == 8 ? 2 : 3));    // log2(32/RB)
     constexpr int WARPS = THREADS / 32;
     static_assert(RB == 4 || RB == 8 || RB == 16 || RB == 32, "RB");
     static_assert(THREADS == 256 || (THREADS == 512 && RB * CHUNKS <= 16), "512 threads leave 128 registers per thread");
     static_assert(RB * CHUNKS <= 32, "register budget");
+    static_assert(EXTRA >= 0 && EXTRA <= 2, "EXTRA");
     extern __shared__ __align__(16) unsigned char smem_raw[];
     cg::cluster_group cluster = cg::this_cluster();
 
@@ -177,7 +181,7 @@ __global__ void __launch_bounds__(THREADS, 1) persistent_kernel(const PersistPar
     const i64 q = (m_i + C - 1) / C;
     const i64 r0 = min(w_r0 + (i64)crank * q, w_r1), r1 = min(r0 + q, w_r1);
     const int rows = (int)(r1 - r0);
-    const int nbatch = (rows + RB - 1) / RB;
+    const int nbatch = (rows + RBT - 1) / RBT;
 
     // The launch must really have put C blocks into each cluster; otherwise nobody would send partials.
     if ((int)cluster.num_blocks() != C) {
@@ -206,22 +210,31 @@ __global__ void __launch_bounds__(THREADS, 1) persistent_kernel(const PersistPar
 
     // REG source: the (single) batch of this warp lives in registers for the whole kernel.
     float4 a[RB][CHUNKS];
-    float y_reg = 0.f;
+    float4 ax[EXTRA > 0 ? EXTRA : 1][CHUNKS];
+    float y_reg = 0.f, y_ext[EXTRA > 0 ? EXTRA : 1];
+    auto load_row = [&](int row, int cs) {
+        const int c = lane + 32 * cs;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (row < rows && c < chunks) {
+            if (SRC == PK_SRC_SMEM) v = reinterpret_cast<const float4*>(slice)[row * chunks + c];
+            else v = __ldg(reinterpret_cast<const float4*>(p.A + (r0 + row) * (i64)ld) + c);
+        }
+        return v;
+    };
     auto load_batch = [&](int b) {
-        const int rb0 = b * RB;
+        const int rb0 = b * RBT;
+#pragma unroll
+        for (int e = 0; e < EXTRA; ++e) {
+            const int row = rb0 + RB + e;
+#pragma unroll
+            for (int cs = 0; cs < CHUNKS; ++cs) ax[e][cs] = load_row(row, cs);
+            y_ext[e] = row < rows ? __ldg(p.y + r0 + row) : 0.f;
+        }
 #pragma unroll
         for (int r = 0; r < RB; ++r) {
             const int row = rb0 + r;
 #pragma unroll
-            for (int cs = 0; cs < CHUNKS; ++cs) {
-                const int c = lane + 32 * cs;
-                float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (row < rows && c < chunks) {
-                    if (SRC == PK_SRC_SMEM) v = reinterpret_cast<const float4*>(slice)[row * chunks + c];
-                    else v = __ldg(reinterpret_cast<const float4*>(p.A + (r0 + row) * (i64)ld) + c);
-                }
-                a[r][cs] = v;
-            }
+            for (int cs = 0; cs < CHUNKS; ++cs) a[r][cs] = load_row(row, cs);
         }
         const int myrow = rb0 + (lane >> SH);
         y_reg = myrow < rows ? __ldg(p.y + r0 + myrow) : 0.f;
@@ -278,6 +291,17 @@ __global__ void __launch_bounds__(THREADS, 1) persistent_kernel(const PersistPar
 #pragma unroll
                     for (int cs = 0; cs < CHUNKS; ++cs) acc[cs] = fma4(pr, a[r][cs], acc[cs]);
                 }
+#pragma unroll
+                for (int e = 0; e < EXTRA; ++e) {
+                    float ze = 0.f;
+#pragma unroll
+                    for (int cs = 0; cs < CHUNKS; ++cs) ze = dot4(ax[e][cs], xr[cs], ze);
+#pragma unroll
+                    for (int off = 16; off >= 1; off >>= 1) ze += __shfl_xor_sync(0xffffffffu, ze, off);
+                    const float pe = loss_residual(p.objective, y_ext[e], ze);      // 0 for a row past the end (y = 0, a = 0)
+#pragma unroll
+                    for (int cs = 0; cs < CHUNKS; ++cs) acc[cs] = fma4(pe, ax[e][cs], acc[cs]);
+                }
             }
 #pragma unroll
             for (int cs = 0; cs < CHUNKS; ++cs) {
@@ -331,20 +355,25 @@ __global__ void __launch_bounds__(THREADS, 1) persistent_kernel(const PersistPar
                 __syncthreads();
                 if (rank_select) {
                     // larger k: every coordinate counts the entries that precede it in (|v| descending, index
-                    // ascending) order; the k entries of rank < k are the message
-                    for (int j = tid; j < ld; j += THREADS) {
-                        unsigned char chosen = 0;
+                    // ascending) order; the k entries of rank < k are the message.  `split` adjacent lanes share a
+                    // coordinate, each counts a contiguous part of the entries, a butterfly adds the parts up.
+                    const int split = (ld * 4 <= THREADS) ? 4 : ((ld * 2 <= THREADS) ? 2 : 1);
+                    const int part_len = (p.d + split - 1) / split;
+                    for (int j0 = 0; j0 < ld; j0 += THREADS / split) {       // uniform trip count: all lanes reach the shuffles
+                        const int j = j0 + tid / split, q = tid % split;
+                        int rank = 0;
                         if (j < p.d) {
                             const unsigned kj = mag_key(vs[j]);
-                            int rank = 0;
+                            const int i1 = min((q + 1) * part_len, p.d);
 #pragma unroll 4
-                            for (int i = 0; i < p.d; ++i) {
+                            for (int i = q * part_len; i < i1; ++i) {
                                 const unsigned ki = mag_key(vs[i]);
                                 rank += (ki > kj || (ki == kj && i < j)) ? 1 : 0;
                             }
-                            chosen = rank < p.k ? 1 : 0;
                         }
-                        sel[j] = chosen;
+                        if (split >= 2) rank += __shfl_xor_sync(0xffffffffu, rank, 1);
+                        if (split >= 4) rank += __shfl_xor_sync(0xffffffffu, rank, 2);
+                        if (q == 0 && j < ld) sel[j] = (j < p.d && rank < p.k) ? 1 : 0;
                     }
                     __syncthreads();
                 }
@@ -431,17 +460,19 @@ __global__ void __launch_bounds__(THREADS, 1) persistent_kernel(const PersistPar
             }
 
             // 5. gather all n*k message words of this epoch (bounded spin)
-            for (int u = tid; u < nmsg; u += THREADS) {
+            auto poll_word = [&](int u, unsigned long long& w) {
                 unsigned spins = 0;
-                unsigned long long w;
-                bool got = true;
                 while (true) {
                     w = ld_relaxed_u64(slot + u);
-                    if ((unsigned)(w >> 48) == epoch) break;
+                    if ((unsigned)(w >> 48) == epoch) return true;
                     ++spins;
-                    if ((spins & 1023u) == 0u && ld_relaxed_u32(p.status) != 0u) { abort_flag = 1; got = false; break; }
-                    if (spins > p.spin_limit) { record_error(p.status, (unsigned)5 /* EF21_ERR_TIMEOUT */); abort_flag = 1; got = false; break; }
+                    if ((spins & 1023u) == 0u && ld_relaxed_u32(p.status) != 0u) { abort_flag = 1; return false; }
+                    if (spins > p.spin_limit) { record_error(p.status, (unsigned)5 /* EF21_ERR_TIMEOUT */); abort_flag = 1; return false; }
                 }
+            };
+            for (int u = tid; u < nmsg; u += THREADS) {
+                unsigned long long w;
+                const bool got = poll_word(u, w);
                 if (p.use_table) {
                     const unsigned idx = (unsigned)(w >> 32) & 0xffffu;
                     if (got && idx < (unsigned)ld) table[(int)(((unsigned)u * k_magic) >> 16) * ld + (int)idx] = (unsigned)w;
