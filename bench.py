@@ -2,7 +2,7 @@
 """Benchmark of the EF21 hot path (libef21) on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload all|headline|stress] [--stress-n N] [--no-cpu] [--no-e2e]
+                    [--workload all|headline|stress|hbm] [--stress-n N] [--no-cpu] [--no-e2e]
 
 A "step" is one EF21 iteration (Algorithm 2's loop body over all n workers).  The headline
 workload is the mushrooms-shaped logistic problem (n = 20, d = 112, N = 8,124, Top-1, gamma = 1/L);
@@ -281,6 +281,31 @@ def run_ours(args):
         return {"ms": ms, "launches": launches, "status": status, "f_end": f_end, "path": h.last_path,
                 "shape": h.get_persistent_shape(), "clocks": sampler.summary() if sampler else None, "handle": h}
 
+    def time_hbm_scale(steps, warmup):
+        wb = inputs.hbm_scale_logistic()
+        rr = time_logistic(wb, wb.k, steps, warmup)
+        b = logistic_bytes_per_iteration(wb.n, wb.d, wb.k, wb.N)
+        gbs = b * steps / (rr["ms"] * 1e-3) / 1e9
+        return {"workload": f"{wb.name}: n={wb.n} d={wb.d} N={wb.N} Top-{wb.k} ({4 * wb.N * wb.d / 1e6:.0f} MB of shards, "
+                            "streamed from HBM every iteration)",
+                "iterations_per_s": steps / (rr["ms"] * 1e-3), "us_per_iteration": rr["ms"] / steps * 1e3, "steps": steps,
+                "algorithmic_bytes_per_iteration": b, "algorithmic_GBps": gbs, "frac_of_hbm_peak": gbs / peak,
+                "launches": rr["launches"], "persistent_shape": rr["shape"], "f_end": rr["f_end"], "device_status": rr["status"]}
+
+    if args.workload == "hbm":
+        r = time_hbm_scale(args.steps if args.steps is not None else 50, max(3, args.warmup if args.warmup is not None else 3))
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": world * r["iterations_per_s"], "unit": UNIT, "n_gpus": world,
+                              "steps": r["steps"], "ms_per_step": r["us_per_iteration"] / 1e3, "dtype": "f32",
+                              "data": "synthetic", "config": {"workload": r["workload"]},
+                              "roofline": {"bound": "hbm", "achieved": r["algorithmic_GBps"], "peak": peak, "unit": "GB/s",
+                                           "frac": r["frac_of_hbm_peak"], "traffic": None, "peak_kind": f"of {peak_kind}",
+                                           "kernel": "persistent_kernel, rows streamed from global memory"},
+                              "gpu_launches": r["launches"], "persistent_shape": r["persistent_shape"]}), flush=True)
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
     # ---- headline ---------------------------------------------------------------------------
     w = inputs.config(HEADLINE)
     steps = args.steps if args.steps is not None else w.T
@@ -352,6 +377,7 @@ def run_ours(args):
                            "us_per_iteration": rr["ms"] / wk.T * 1e3, "algorithmic_GBps": gbs, "frac_of_hbm_peak": gbs / peak,
                            "launches": rr["launches"], "persistent_shape": rr["shape"], "f_end": rr["f_end"]})
         others.append(time_stress(None, 50, 3))
+        others.append(time_hbm_scale(50, 3))
         # EF21+ (Algorithm 3) on the headline shapes: launch-per-stage kernels, two Top-k per worker and step
         wp = inputs.config(HEADLINE)
         rp = time_logistic(wp, wp.k, 500, 10, variant=B.VARIANT_EF21_PLUS)
@@ -371,9 +397,10 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="all", choices=["all", "headline", "stress"],
+    ap.add_argument("--workload", default="all", choices=["all", "headline", "stress", "hbm"],
                     help="all: headline line with the other workloads attached; headline: only the headline; "
-                         "stress: only the supplied-gradient workload (its own line; for profiling)")
+                         "stress: only the supplied-gradient workload; hbm: only the logistic workload whose shards "
+                         "exceed L2 (each its own line; for profiling)")
     ap.add_argument("--stress-n", type=int, default=None, help="workers of the stress workload (default 64)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end timing")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle timing")

@@ -201,6 +201,14 @@ def config(index: int, k: Optional[int] = None, scale: float = 1.0):
     raise ValueError(f"no workload {index}")
 
 
+def hbm_scale_logistic(N: int = 500_000):
+    """Rows shaped like workload 3 (d = 300, Bernoulli(0.04) features, planted labels with 5 % flips, n = 20 equal
+    shards) but N of them, so that the shards (4*N*300 bytes; 600 MB by default) no longer fit in L2 and every
+    iteration streams them from HBM.  Same generator and stepsize rule as the other logistic workloads."""
+    return make_logistic("w8a-shaped rows beyond L2", n=20, d=300, N=N, k=1, seed=5, features="bernoulli",
+                         density=0.04, flip=0.05, T=50)
+
+
 def minibatch_rows(seed: int, step: int, row_offsets: np.ndarray, tau: int) -> np.ndarray:
     """Rows of one stochastic step: for every worker tau distinct row numbers inside its shard (sampling
     without replacement, as in the paper's minibatch experiments), int32 [n, tau], from its own stream."""
