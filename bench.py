@@ -2,7 +2,7 @@
 """Benchmark of the EF21 hot path (libef21) on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload all|headline|stress|hbm] [--stress-n N] [--no-cpu] [--no-e2e]
+                    [--workload all|headline|stress|hbm] [--path auto|launches|persistent] [--stress-n N] [--no-cpu] [--no-e2e]
 
 A "step" is one EF21 iteration (Algorithm 2's loop body over all n workers).  The headline
 workload is the mushrooms-shaped logistic problem (n = 20, d = 112, N = 8,124, Top-1, gamma = 1/L);
@@ -246,6 +246,8 @@ def run_ours(args):
     def time_logistic(w, k, steps, warmup, repeats=3, with_clocks=False, variant=0):
         h = B.EF21(w.n, w.d, k, w.gamma, w.lam, total_rows=w.N, device=device)
         h.set_variant(variant)
+        if variant == 0:
+            h.set_path({"auto": B.PATH_AUTO, "launches": B.PATH_LAUNCHES, "persistent": B.PATH_PERSISTENT}[args.path])
         h.load_shards(dev(w.A), dev(w.y), w.row_offsets)
         h.init(B.INIT_COMPRESSED)
         x0, g0, gi0, _, _ = h.get_state()
@@ -300,7 +302,8 @@ def run_ours(args):
                               "data": "synthetic", "config": {"workload": r["workload"]},
                               "roofline": {"bound": "hbm", "achieved": r["algorithmic_GBps"], "peak": peak, "unit": "GB/s",
                                            "frac": r["frac_of_hbm_peak"], "traffic": None, "peak_kind": f"of {peak_kind}",
-                                           "kernel": "persistent_kernel, rows streamed from global memory"},
+                                           "kernel": "persistent_kernel, rows streamed from global memory" if args.path != "launches"
+                                                     else "grad_stream_kernel (dominant) + per-stage kernels"},
                               "gpu_launches": r["launches"], "persistent_shape": r["persistent_shape"]}), flush=True)
         if world > 1:
             dist.destroy_process_group()
@@ -401,6 +404,8 @@ def main():
                     help="all: headline line with the other workloads attached; headline: only the headline; "
                          "stress: only the supplied-gradient workload; hbm: only the logistic workload whose shards "
                          "exceed L2 (each its own line; for profiling)")
+    ap.add_argument("--path", default="auto", choices=["auto", "launches", "persistent"],
+                    help="execution path of the logistic workloads (default: the library's own choice)")
     ap.add_argument("--stress-n", type=int, default=None, help="workers of the stress workload (default 64)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end timing")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle timing")

@@ -170,8 +170,9 @@ ef21_status ef21_topk(const float* v_dev, int32_t batch, int64_t d, int32_t k,
  * library routine.
  *
  * Limits: batch <= 64 and batch * ceil(d / 4096) <= 16384 (e.g. 64 vectors of 2^20 entries, or
- * one of 2^26); beyond that the call returns EF21_ERR_UNSUPPORTED and does nothing.  Always
- * runs the multi-pass radix select.
+ * one of 2^26); beyond that the call returns EF21_ERR_UNSUPPORTED and does nothing.  Vectors
+ * of up to 8,192 entries take the one-launch kernel (which needs no scratch), longer ones the
+ * multi-pass radix select.
  * The first call on a device looks up the device address of the scratch array
  * (cudaGetSymbolAddress, with that device current) and caches it; make that first call outside
  * of any stream capture.

@@ -62,8 +62,25 @@ TopkLayout topk_layout(i64 batch, i64 d, i64 k) {
     return L;
 }
 
+typedef void (*GradTileKernel)(const float*, const float*, const float*, const RowTile*, int, int, float*, double*,
+                               const int*, int, const i64*, unsigned*);
+
+// The one-read gradient kernel for rows of up to 1,024 columns (chunk slots = float4 per lane and row); wider
+// rows use the two-sweep kernel.
+GradTileKernel grad_stream_lookup(i64 ld) {
+    const i64 slots = (ld / 4 + 31) / 32;
+    if (slots <= 1) return grad_stream_kernel<1, 16>;
+    if (slots == 2) return grad_stream_kernel<2, 8>;
+    if (slots == 3) return grad_stream_kernel<3, 4>;
+    if (slots == 4) return grad_stream_kernel<4, 4>;
+    if (slots <= 6) return grad_stream_kernel<6, 2>;
+    if (slots <= 8) return grad_stream_kernel<8, 2>;
+    return nullptr;
+}
+
 int grad_tile_rows(i64 N, i64 ld) {
-    i64 cap = 65536 / (ld * 4);
+    // two-sweep kernel: a tile's rows should stay in L1 for the second sweep; one-read kernel: any size
+    i64 cap = grad_stream_lookup(ld) ? GRAD_TILE_MAX_ROWS : 65536 / (ld * 4);
     if (cap < 1) cap = 1;
     if (cap > GRAD_TILE_MAX_ROWS) cap = GRAD_TILE_MAX_ROWS;
     i64 want = ceil_div(N, 4 * 148);
@@ -243,6 +260,13 @@ ef21_status enqueue_topk_fast(cudaStream_t st, const float* a, i64 pitch_a, cons
 ef21_status enqueue_topk_general(cudaStream_t st, const float* a, i64 pitch_a, const float* b, i64 pitch_b,
                                  int batch, i64 d, int k, int* idx_out, float* val_out,
                                  const TopkBuffers& B, i64* launches) {
+    if (d <= TKS_MAX_D) {
+        // short vectors: the whole selection in one launch, one block per vector (no scratch)
+        tk_small_kernel<<<batch, TKS_BLOCK, (size_t)d * 4, st>>>(a, pitch_a, b, pitch_b, (int)d, k, idx_out, val_out);
+        if (launches) *launches += 1;
+        CU(cudaGetLastError());
+        return EF21_OK;
+    }
     tk_reset_kernel<<<batch, 256, 0, st>>>(B.state, B.hist, batch, (unsigned)k);
     dim3 grid((unsigned)B.nchunks, (unsigned)batch);
     for (int level = 0; level < 3; ++level) {
@@ -260,16 +284,23 @@ ef21_status enqueue_topk_general(cudaStream_t st, const float* a, i64 pitch_a, c
 
 ef21_status enqueue_grads(ef21_ctx* c, bool with_loss) {
     if (c->num_tiles > 0) {
-        grad_tiles_kernel<<<c->num_tiles, GRAD_BLOCK, 0, c->stream>>>(
-            c->at<float>(c->L.A), c->at<float>(c->L.y), c->x(), c->at<RowTile>(c->L.tiles), (int)c->L.ld, c->objective,
-            c->at<float>(c->L.partial), with_loss ? c->at<double>(c->L.loss_partial) : nullptr, nullptr, 0,
-            c->at<i64>(c->L.row_off), c->status());
+        GradTileKernel stream = grad_stream_lookup(c->L.ld);
+        if (stream)
+            stream<<<c->num_tiles, GRAD_STREAM_BLOCK, (size_t)(GRAD_STREAM_BLOCK / 32) * c->L.ld * 4, c->stream>>>(
+                c->at<float>(c->L.A), c->at<float>(c->L.y), c->x(), c->at<RowTile>(c->L.tiles), (int)c->L.ld, c->objective,
+                c->at<float>(c->L.partial), with_loss ? c->at<double>(c->L.loss_partial) : nullptr, nullptr, 0,
+                c->at<i64>(c->L.row_off), c->status());
+        else
+            grad_tiles_kernel<<<c->num_tiles, GRAD_BLOCK, 0, c->stream>>>(
+                c->at<float>(c->L.A), c->at<float>(c->L.y), c->x(), c->at<RowTile>(c->L.tiles), (int)c->L.ld, c->objective,
+                c->at<float>(c->L.partial), with_loss ? c->at<double>(c->L.loss_partial) : nullptr, nullptr, 0,
+                c->at<i64>(c->L.row_off), c->status());
         c->launches += 1;
     }
-    dim3 grid((unsigned)ceil_div(c->L.ld, 256), (unsigned)c->n);
-    grad_finish_kernel<<<grid, 256, 0, c->stream>>>(c->at<float>(c->L.partial), c->at<int>(c->L.tile_begin),
-                                                    c->at<i64>(c->L.row_off), c->x(), c->lambda, (int)c->d,
-                                                    (int)c->L.ld, c->at<float>(c->L.grad), 0);
+    dim3 grid((unsigned)ceil_div(c->L.ld, GRAD_FINISH_COLS), (unsigned)c->n);
+    grad_finish_kernel<<<grid, GRAD_FINISH_COLS * GRAD_FINISH_LANES, 0, c->stream>>>(
+        c->at<float>(c->L.partial), c->at<int>(c->L.tile_begin), c->at<i64>(c->L.row_off), c->x(), c->lambda, (int)c->d,
+        (int)c->L.ld, c->at<float>(c->L.grad), 0);
     c->launches += 1;
     CU(cudaGetLastError());
     return EF21_OK;
@@ -297,13 +328,19 @@ ef21_status enqueue_minibatch_grads(ef21_ctx* c, const int* batch_dev, int tau) 
         CU(cudaStreamSynchronize(c->stream));      // the host vectors may be rebuilt by the next call
         c->mb_tau = tau;
     }
-    grad_tiles_kernel<<<(unsigned)c->mb_tiles.size(), GRAD_BLOCK, 0, c->stream>>>(
-        c->at<float>(c->L.A), c->at<float>(c->L.y), c->x(), c->at<RowTile>(c->L.mb_tiles), (int)c->L.ld, c->objective,
-        c->at<float>(c->L.partial), nullptr, batch_dev, tau, c->at<i64>(c->L.row_off), c->status());
-    dim3 grid((unsigned)ceil_div(c->L.ld, 256), (unsigned)c->n);
-    grad_finish_kernel<<<grid, 256, 0, c->stream>>>(c->at<float>(c->L.partial), c->at<int>(c->L.mb_tile_begin),
-                                                    c->at<i64>(c->L.row_off), c->x(), c->lambda, (int)c->d,
-                                                    (int)c->L.ld, c->at<float>(c->L.grad), tau);
+    GradTileKernel stream = grad_stream_lookup(c->L.ld);
+    if (stream)
+        stream<<<(unsigned)c->mb_tiles.size(), GRAD_STREAM_BLOCK, (size_t)(GRAD_STREAM_BLOCK / 32) * c->L.ld * 4, c->stream>>>(
+            c->at<float>(c->L.A), c->at<float>(c->L.y), c->x(), c->at<RowTile>(c->L.mb_tiles), (int)c->L.ld, c->objective,
+            c->at<float>(c->L.partial), nullptr, batch_dev, tau, c->at<i64>(c->L.row_off), c->status());
+    else
+        grad_tiles_kernel<<<(unsigned)c->mb_tiles.size(), GRAD_BLOCK, 0, c->stream>>>(
+            c->at<float>(c->L.A), c->at<float>(c->L.y), c->x(), c->at<RowTile>(c->L.mb_tiles), (int)c->L.ld, c->objective,
+            c->at<float>(c->L.partial), nullptr, batch_dev, tau, c->at<i64>(c->L.row_off), c->status());
+    dim3 grid((unsigned)ceil_div(c->L.ld, GRAD_FINISH_COLS), (unsigned)c->n);
+    grad_finish_kernel<<<grid, GRAD_FINISH_COLS * GRAD_FINISH_LANES, 0, c->stream>>>(
+        c->at<float>(c->L.partial), c->at<int>(c->L.mb_tile_begin), c->at<i64>(c->L.row_off), c->x(), c->lambda, (int)c->d,
+        (int)c->L.ld, c->at<float>(c->L.grad), tau);
     c->launches += 2;
     CU(cudaGetLastError());
     return EF21_OK;

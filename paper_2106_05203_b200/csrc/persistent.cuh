@@ -106,34 +106,6 @@ __device__ __forceinline__ void st_async_f4(unsigned remote_dst, float4 v, unsig
                  ::"r"(remote_dst), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "r"(remote_bar) : "memory");
 }
 
-// Sum of v[r] over the 32 lanes for RB rows at once: after the call lane L holds the total of
-// row L / (32/RB).  RB-1 shuffles for the halving steps plus log2(32/RB) butterfly steps.
-template <int RB>
-__device__ __forceinline__ float reduce_rows(float (&v)[RB], int lane) {
-#pragma unroll
-    for (int half = RB / 2, off = 16; half >= 1; half >>= 1, off >>= 1) {
-        const bool upper = (lane & off) != 0;
-#pragma unroll
-        for (int r = 0; r < half; ++r) {
-            const float keep = upper ? v[r + half] : v[r];
-            const float send = upper ? v[r] : v[r + half];
-            v[r] = keep + __shfl_xor_sync(0xffffffffu, send, off);
-        }
-    }
-    float s = v[0];
-#pragma unroll
-    for (int off = (32 / RB) / 2; off >= 1; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
-    return s;
-}
-
-__device__ __forceinline__ float4 fma4(float s, float4 a, float4 c) {
-    c.x = fmaf(s, a.x, c.x); c.y = fmaf(s, a.y, c.y); c.z = fmaf(s, a.z, c.z); c.w = fmaf(s, a.w, c.w);
-    return c;
-}
-__device__ __forceinline__ float dot4(float4 a, float4 b, float z) {
-    z = fmaf(a.x, b.x, z); z = fmaf(a.y, b.y, z); z = fmaf(a.z, b.z, z); z = fmaf(a.w, b.w, z);
-    return z;
-}
 __device__ __forceinline__ float comp_of(const float4& v, int c) {
     return c == 0 ? v.x : (c == 1 ? v.y : (c == 2 ? v.z : v.w));
 }

@@ -196,4 +196,91 @@ tk_write_kernel(const float* __restrict__ a, i64 pitch_a, const float* __restric
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Short vectors (d <= TKS_MAX_D): the whole selection in ONE launch, one block per vector.
+//   v = a - b is formed once into shared memory; radix select on the 31-bit key with digits of
+//   8 + 8 + 8 + 7 bits (shared-memory histogram over the entries that match the prefix, warp 0
+//   locates the digit that holds the k-th largest key); every thread then owns a contiguous piece of
+//   the vector, counts its entries above the threshold key T and equal to it, one block scan turns
+//   the counts into output positions (ties are taken in index order until need_ties are used up),
+//   and the pairs are written in ascending index order.
+// ---------------------------------------------------------------------------------------------
+constexpr int TKS_MAX_D = 8192;
+constexpr int TKS_BLOCK = 512;
+
+__global__ void __launch_bounds__(TKS_BLOCK)
+tk_small_kernel(const float* __restrict__ a, i64 pitch_a, const float* __restrict__ b, i64 pitch_b,
+                int d, int k, int* __restrict__ idx_out, float* __restrict__ val_out) {
+    extern __shared__ __align__(16) unsigned char tks_smem[];
+    float* vs = reinterpret_cast<float*>(tks_smem);                     // [d]
+    __shared__ unsigned hist[256];
+    __shared__ unsigned scan_scratch[33];
+    __shared__ unsigned sh_prefix, sh_need;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const float* __restrict__ av = a + (i64)blockIdx.x * pitch_a;
+    const float* __restrict__ bv = b ? b + (i64)blockIdx.x * pitch_b : nullptr;
+    for (int j = tid; j < d; j += TKS_BLOCK) vs[j] = diff_at(av, bv, j);
+    if (tid == 0) { sh_prefix = 0u; sh_need = (unsigned)k; }
+    // radix select: after the four digits sh_prefix is the k-th largest key T and sh_need the number of
+    // entries equal to T that belong to the Top-k
+#pragma unroll 1
+    for (int pass = 0; pass < 4; ++pass) {
+        const int shift = pass == 0 ? 23 : (pass == 1 ? 15 : (pass == 2 ? 7 : 0));
+        const int bits = pass == 3 ? 7 : 8;
+        if (tid < 256) hist[tid] = 0u;
+        __syncthreads();
+        const unsigned prefix = sh_prefix;
+        for (int j = tid; j < d; j += TKS_BLOCK) {
+            const unsigned key = mag_key(vs[j]);
+            if ((key >> (shift + bits)) == prefix) atomicAdd(&hist[(key >> shift) & ((1u << bits) - 1u)], 1u);
+        }
+        __syncthreads();
+        if (warp == 0) {
+            // lane 0 owns the top eight bins, lane 31 the lowest eight; walk down until `need` is covered
+            const unsigned need = sh_need;
+            unsigned c[8], sum = 0u;
+#pragma unroll
+            for (int q = 0; q < 8; ++q) { c[q] = hist[255 - (8 * lane + q)]; sum += c[q]; }
+            const unsigned incl = warp_incl_scan(sum), excl = incl - sum;
+            if (excl < need && need <= incl) {
+                unsigned rest = need - excl;
+                int bin = 0;
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    if (rest != 0u) {
+                        if (c[q] >= rest) { bin = 255 - (8 * lane + q); sh_need = rest; rest = 0u; }
+                        else rest -= c[q];
+                    }
+                }
+                sh_prefix = (prefix << bits) | (unsigned)bin;
+            }
+        }
+        __syncthreads();
+    }
+    const unsigned T = sh_prefix, need_ties = sh_need;
+    // contiguous piece per thread, so that thread order is index order
+    const int seg = (d + TKS_BLOCK - 1) / TKS_BLOCK;
+    const int j0 = min(tid * seg, d), j1 = min(j0 + seg, d);
+    unsigned gt = 0u, eq = 0u;
+    for (int j = j0; j < j1; ++j) {
+        const unsigned key = mag_key(vs[j]);
+        gt += key > T ? 1u : 0u;
+        eq += key == T ? 1u : 0u;
+    }
+    unsigned total;
+    const unsigned before = block_excl_scan((gt << 16) | eq, scan_scratch, total);     // counts <= 8192 each
+    unsigned eq_before = before & 0xffffu;
+    const unsigned gt_before = before >> 16;
+    unsigned pos = gt_before + min(eq_before, need_ties);
+    int* __restrict__ io = idx_out + (i64)blockIdx.x * k;
+    float* __restrict__ vo = val_out + (i64)blockIdx.x * k;
+    for (int j = j0; j < j1; ++j) {
+        const float v = vs[j];
+        const unsigned key = mag_key(v);
+        bool take = key > T;
+        if (key == T) { take = eq_before < need_ties; ++eq_before; }
+        if (take) { io[pos] = j; vo[pos] = v; ++pos; }
+    }
+}
+
 }  // namespace ef21

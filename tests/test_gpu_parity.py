@@ -104,6 +104,48 @@ def test_local_gradients_uneven_and_empty_shards(B, oracle32):
         assert rel_l2(got[i], want[i]) <= 1e-5
 
 
+@pytest.mark.parametrize("d", [1, 5, 127, 128, 129, 256, 300, 384, 500, 513, 700, 768, 1000, 1024, 1025, 1500])
+def test_local_gradients_every_row_width(d, B, oracle32):
+    # launch-per-stage gradient kernels: each register layout of the one-read kernel (up to 1,024 columns,
+    # full and ragged last chunk), the two-sweep kernel beyond, ragged tiles (shards of 1, 7, 300 and 611 rows
+    # and an empty one), loss and gradients
+    rng = np.random.default_rng(1000 + d)
+    off = np.array([0, 1, 8, 8, 308, 919], dtype=np.int64)
+    n, N = len(off) - 1, int(off[-1])
+    A = rng.standard_normal((N, d)).astype(np.float32) / np.float32(np.sqrt(d))
+    y = np.where(rng.random(N) < 0.5, -1.0, 1.0).astype(np.float32)
+    x = (rng.standard_normal(d) * 0.5).astype(np.float32)
+    lam = 0.1
+    h = B.EF21(n, d, 1, 0.1, lam, total_rows=N)
+    h.set_path(B.PATH_LAUNCHES)
+    h.load_shards(dev(A), dev(y), off)
+    h.set_x(dev(x))
+    got = h.local_grads().cpu().numpy()
+    want = oracle32.all_grads(A, y, off, x, lam)
+    for i in range(n):
+        assert rel_l2(got[i], want[i]) <= 1e-5, (d, i)
+    h.init(B.INIT_ZERO)
+    assert h.eval()[0] == pytest.approx(oracle32.loss(A, y, off, x, lam), rel=1e-6)
+    assert h.poll() == 0
+
+
+@pytest.mark.parametrize("d,k", [(1, 1), (2, 1), (300, 1), (300, 300), (511, 7), (512, 512), (513, 64), (4097, 40),
+                                 (8191, 8191), (8192, 1), (8192, 300), (8193, 300)])
+def test_topk_short_vectors_one_launch(d, k, B, oracle32):
+    # the one-launch kernel (up to 8,192 entries) and the first size beyond it, on heavy ties: quantised
+    # values, blocks of equal magnitude with both signs, zeros of both signs
+    rng = np.random.default_rng(d * 31 + k)
+    V = (np.round(rng.standard_normal((3, d)) * 4) / 4).astype(np.float32)
+    V[1, ::3] = np.float32(-0.0)
+    V[2] = np.where(rng.random(d) < 0.5, np.float32(1.5), np.float32(-1.5))
+    idx, val = B.topk(dev(V), k)
+    idx, val = idx.cpu().numpy(), val.cpu().numpy()
+    for i in range(3):
+        wi, wv = oracle32.topk(V[i], k)
+        np.testing.assert_array_equal(idx[i], wi)
+        np.testing.assert_array_equal(val[i].view(np.uint32), wv.view(np.uint32))
+
+
 def test_eval_matches_oracle(B, oracle32):
     w = inputs.config(0)
     h = make_gpu(w); h.init(B.INIT_COMPRESSED); h.step(5)
