@@ -157,6 +157,7 @@ struct ef21_ctx {
     int num_tiles;
     int path, last_path;
     bool agg_off_ready;                 // the last selection already wrote the aggregation's tile offsets
+    bool agg_off_static;                // one tile only: the offsets are (0, k) whatever the messages; written once
     int pk_cluster, pk_rb, pk_src, pk_threads;      // forced persistent-kernel shape (0 / -1 = automatic)
     int pk_used_cluster, pk_used_rb, pk_used_src, pk_used_threads;
     unsigned spin_limit;
@@ -259,10 +260,15 @@ ef21_status enqueue_topk_fast(cudaStream_t st, const float* a, i64 pitch_a, cons
 // Exact Top-k of v = a - b for `batch` vectors (b may be null); general multi-block path.
 ef21_status enqueue_topk_general(cudaStream_t st, const float* a, i64 pitch_a, const float* b, i64 pitch_b,
                                  int batch, i64 d, int k, int* idx_out, float* val_out,
-                                 const TopkBuffers& B, i64* launches) {
+                                 const TopkBuffers& B, i64* launches, float* apply_to = nullptr, i64 pitch_apply = 0,
+                                 bool* applied = nullptr) {
+    if (applied) *applied = false;
     if (d <= TKS_MAX_D) {
-        // short vectors: the whole selection in one launch, one block per vector (no scratch)
-        tk_small_kernel<<<batch, TKS_BLOCK, (size_t)d * 4, st>>>(a, pitch_a, b, pitch_b, (int)d, k, idx_out, val_out);
+        // short vectors: the whole selection in one launch, one block per vector (no scratch); the same
+        // launch adds the messages to apply_to if the caller asks for it
+        tk_small_kernel<<<batch, TKS_BLOCK, (size_t)d * 4, st>>>(a, pitch_a, b, pitch_b, (int)d, k, idx_out, val_out,
+                                                                 apply_to, pitch_apply);
+        if (applied) *applied = apply_to != nullptr;
         if (launches) *launches += 1;
         CU(cudaGetLastError());
         return EF21_OK;
@@ -357,12 +363,15 @@ ef21_status enqueue_round_select(ef21_ctx* c, const float* a, i64 pitch_a, bool 
         c->agg_off_ready = true;
     } else {
         c->agg_off_ready = false;
+        bool applied = false;
         EF(enqueue_topk_general(c->stream, a, pitch_a, c->gi(), c->L.ld, c->n, c->d, c->k, c->msg_idx(),
-                                c->msg_val(), B, &c->launches));
-        const i64 total = (i64)c->n * c->k;
-        apply_messages_kernel<<<(unsigned)ceil_div(total, 256), 256, 0, c->stream>>>(c->msg_idx(), c->msg_val(), total,
-                                                                                    c->k, c->L.ld, c->gi());
-        c->launches += 1;
+                                c->msg_val(), B, &c->launches, c->gi(), c->L.ld, &applied));
+        if (!applied) {
+            const i64 total = (i64)c->n * c->k;
+            apply_messages_kernel<<<(unsigned)ceil_div(total, 256), 256, 0, c->stream>>>(c->msg_idx(), c->msg_val(), total,
+                                                                                        c->k, c->L.ld, c->gi());
+            c->launches += 1;
+        }
     }
     CU(cudaGetLastError());
     return EF21_OK;
@@ -377,11 +386,12 @@ ef21_status enqueue_round_aggregate(ef21_ctx* c, bool update_x) {
 
 // target_j += factor * (sum over workers, ascending, of the values sent for coordinate j).
 ef21_status enqueue_aggregate_into(ef21_ctx* c, float* target, float factor, bool update_x) {
-    if (!c->agg_off_ready) {
+    if (!c->agg_off_ready && !(c->L.agg_tiles == 1 && c->agg_off_static)) {
         const i64 noff = (i64)c->n * (c->L.agg_tiles + 1);
         agg_offsets_kernel<<<(unsigned)ceil_div(noff, 256), 256, 0, c->stream>>>(c->msg_idx(), c->n, c->k,
                                                                                 c->L.agg_tiles, c->at<int>(c->L.agg_off));
         c->launches += 1;
+        c->agg_off_static = c->L.agg_tiles == 1;
     }
     c->agg_off_ready = false;
     auto kern = c->n <= AGG_STAGE_MAX_N
@@ -733,7 +743,7 @@ ef21_status ef21_create(ef21_ctx** out, int32_t n, int64_t d, int32_t k, float g
     c->L = L;
     c->shards_loaded = false; c->inited = false; c->num_tiles = 0;
     c->path = EF21_PATH_AUTO; c->last_path = 0; c->launches = 0;
-    c->pk_cluster = 0; c->pk_rb = 0; c->pk_src = -1; c->pk_threads = 0; c->agg_off_ready = false;
+    c->pk_cluster = 0; c->pk_rb = 0; c->pk_src = -1; c->pk_threads = 0; c->agg_off_ready = false; c->agg_off_static = false;
     c->pk_used_cluster = c->pk_used_rb = 0; c->pk_used_src = -1; c->pk_used_threads = 0;
     c->spin_limit = 1u << 22;
     c->force_general_topk = false;

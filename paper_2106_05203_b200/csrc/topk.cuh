@@ -203,14 +203,15 @@ tk_write_kernel(const float* __restrict__ a, i64 pitch_a, const float* __restric
 //   locates the digit that holds the k-th largest key); every thread then owns a contiguous piece of
 //   the vector, counts its entries above the threshold key T and equal to it, one block scan turns
 //   the counts into output positions (ties are taken in index order until need_ties are used up),
-//   and the pairs are written in ascending index order.
+//   and the pairs are written in ascending index order.  apply_to (optional): the vector that receives
+//   g_i + c_i on the selected coordinates in the same launch.
 // ---------------------------------------------------------------------------------------------
 constexpr int TKS_MAX_D = 8192;
 constexpr int TKS_BLOCK = 512;
 
 __global__ void __launch_bounds__(TKS_BLOCK)
-tk_small_kernel(const float* __restrict__ a, i64 pitch_a, const float* __restrict__ b, i64 pitch_b,
-                int d, int k, int* __restrict__ idx_out, float* __restrict__ val_out) {
+tk_small_kernel(const float* __restrict__ a, i64 pitch_a, const float* b, i64 pitch_b,
+                int d, int k, int* __restrict__ idx_out, float* __restrict__ val_out, float* apply_to, i64 pitch_apply) {
     extern __shared__ __align__(16) unsigned char tks_smem[];
     float* vs = reinterpret_cast<float*>(tks_smem);                     // [d]
     __shared__ unsigned hist[256];
@@ -218,8 +219,8 @@ tk_small_kernel(const float* __restrict__ a, i64 pitch_a, const float* __restric
     __shared__ unsigned sh_prefix, sh_need;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const float* __restrict__ av = a + (i64)blockIdx.x * pitch_a;
-    const float* __restrict__ bv = b ? b + (i64)blockIdx.x * pitch_b : nullptr;
-    for (int j = tid; j < d; j += TKS_BLOCK) vs[j] = diff_at(av, bv, j);
+    const float* bv = b ? b + (i64)blockIdx.x * pitch_b : nullptr;      // may be the vector apply_to updates below
+    for (int j = tid; j < d; j += TKS_BLOCK) vs[j] = bv ? __fsub_rn(av[j], bv[j]) : av[j];
     if (tid == 0) { sh_prefix = 0u; sh_need = (unsigned)k; }
     // radix select: after the four digits sh_prefix is the k-th largest key T and sh_need the number of
     // entries equal to T that belong to the Top-k
@@ -279,7 +280,13 @@ tk_small_kernel(const float* __restrict__ a, i64 pitch_a, const float* __restric
         const unsigned key = mag_key(v);
         bool take = key > T;
         if (key == T) { take = eq_before < need_ties; ++eq_before; }
-        if (take) { io[pos] = j; vo[pos] = v; ++pos; }
+        if (take) {
+            io[pos] = j; vo[pos] = v; ++pos;
+            if (apply_to) {            // g_i <- g_i + c_i on the selected coordinate (Algorithm 2, node loop)
+                float* p = apply_to + (i64)blockIdx.x * pitch_apply + j;
+                *p = __fadd_rn(*p, v);
+            }
+        }
     }
 }
 
