@@ -243,7 +243,7 @@ def run_ours(args):
             dist.destroy_process_group()
         return
 
-    def time_logistic(w, k, steps, warmup, repeats=3, with_clocks=False, variant=0):
+    def time_logistic(w, k, steps, warmup, repeats=5, with_clocks=False, variant=0):
         h = B.EF21(w.n, w.d, k, w.gamma, w.lam, total_rows=w.N, device=device)
         h.set_variant(variant)
         if variant == 0:
@@ -354,7 +354,7 @@ def run_ours(args):
                    "l2": "L2 flushed (256 MB written) before each timed run; inside a run the iterations re-read the same "
                          "shards, which is the method's own access pattern",
                    "replicas": "replicas only: each rank runs the whole n-worker problem" if world > 1 else None,
-                   "timed_runs": 3, "value_from": "median run"},
+                   "timed_runs": 5, "value_from": "median run"},
         "roofline": roofline, "e2e": e2e, "gpu_launches": r["launches"], "clocks": r["clocks"],
         "device_status": r["status"], "f_end": r["f_end"], "persistent_shape": r["shape"],
     }
