@@ -128,7 +128,12 @@ ef21_status ef21_init_grads(ef21_ctx* ctx, const float* V_dev, int32_t mode);
 
 /* `steps` iterations of Algorithm 2's loop (x update, local gradients of Eq. 19,
  * difference, Top-k, g_i update, aggregation).  After init and t steps in total the
- * state is (x^t, g^t, g_i^t) in the paper's indexing. */
+ * state is (x^t, g^t, g_i^t) in the paper's indexing.
+ * On the launch-per-stage path with d <= 8,192 and steps >= 3, the iterations after the first are
+ * replayed as a CUDA graph that the handle captures once (on a stream of its own; the CUDA runtime
+ * keeps the graph's resources until ef21_destroy) and launches into the handle's stream; if that
+ * stream is itself being captured, or the capture fails, the kernels are launched one by one.
+ * Results are identical either way. */
 ef21_status ef21_step(ef21_ctx* ctx, int32_t steps);
 /* The same loop with grad f_i replaced by the caller's V_dev[n][d], re-used unchanged at
  * each of the `steps` iterations (the static input sequence of Section 3.1); call with

@@ -166,6 +166,11 @@ struct ef21_ctx {
     int objective;                      // EF21_OBJECTIVE_*
     cudaStream_t aux_stream;            // created on first use: overlaps the next threshold estimate
     cudaEvent_t ev_fork, ev_join;
+    cudaStream_t cap_stream;            // library-owned stream on which the iteration graph is captured
+    cudaGraphExec_t iter_graph;         // one launch-path iteration of ef21_step, captured on first use
+    int iter_graph_key;                 // what it was captured for (variant, objective)
+    i64 iter_graph_launches;            // kernel launches inside it
+    bool iter_graph_off;                // capture failed once: keep to plain launches
     i64 launches;
     std::vector<i64> row_off;
     std::vector<RowTile> tiles;
@@ -769,6 +774,8 @@ void ef21_destroy(ef21_ctx* ctx) {
     if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
     if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
     if (ctx->aux_stream) cudaStreamDestroy(ctx->aux_stream);
+    if (ctx->iter_graph) cudaGraphExecDestroy(ctx->iter_graph);
+    if (ctx->cap_stream) cudaStreamDestroy(ctx->cap_stream);
     delete ctx;
 }
 
@@ -820,28 +827,80 @@ ef21_status ef21_init_grads(ef21_ctx* c, const float* V_dev, int32_t mode) {
     return init_from(c, V_dev, c->d, mode);
 }
 
+// One iteration of ef21_step on the launch path, as plain kernel launches on the handle's stream.
+static ef21_status enqueue_launch_iteration(ef21_ctx* c) {
+    if (c->variant == EF21_VARIANT_EF) {
+        EF(enqueue_grads(c, false));
+        return enqueue_ef_round(c, c->at<float>(c->L.grad), c->L.ld);
+    }
+    EF(enqueue_x_update(c));
+    EF(enqueue_grads(c, false));
+    if (c->variant == EF21_VARIANT_EF21_PLUS) return enqueue_plus_round(c, c->at<float>(c->L.grad), c->L.ld);
+    return enqueue_round(c, c->at<float>(c->L.grad), c->L.ld, false);
+}
+
+// `steps` launch-path iterations.  Short vectors (the one-launch Top-k) make an iteration a fixed list of
+// five to nine small kernels whose cost is their launches: from the second iteration of a call on, the
+// list is replayed as a CUDA graph captured once per handle and method.  The first iteration always
+// runs as plain launches (it may still write the one-time aggregation offsets).  Anything that stands
+// in the way (the caller's stream is itself being captured, capture or instantiation fails) leaves the
+// plain launches, which give the same results.
+static ef21_status run_launch_iterations(ef21_ctx* c, int steps) {
+    int done = 0;
+    const bool graphable = c->d <= TKS_MAX_D && steps >= 3 && !c->iter_graph_off;
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (graphable && cudaStreamIsCapturing(c->stream, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusNone) {
+        EF(enqueue_launch_iteration(c));
+        done = 1;
+        const int key = c->variant * 16 + c->objective;
+        if (c->iter_graph && c->iter_graph_key != key) { cudaGraphExecDestroy(c->iter_graph); c->iter_graph = nullptr; }
+        if (!c->iter_graph) {
+            const i64 before = c->launches;
+            cudaGraph_t graph = nullptr;
+            // captured on a stream of the library's own (the caller's may be the legacy default stream, which
+            // cannot be captured); the graph is then launched into the caller's stream
+            bool ok = c->cap_stream || cudaStreamCreateWithFlags(&c->cap_stream, cudaStreamNonBlocking) == cudaSuccess;
+            ok = ok && cudaStreamBeginCapture(c->cap_stream, cudaStreamCaptureModeThreadLocal) == cudaSuccess;
+            if (ok) {
+                cudaStream_t user_stream = c->stream;
+                c->stream = c->cap_stream;
+                const ef21_status st = enqueue_launch_iteration(c);
+                c->stream = user_stream;
+                ok = cudaStreamEndCapture(c->cap_stream, &graph) == cudaSuccess && st == EF21_OK && graph != nullptr;
+            }
+            if (ok) ok = cudaGraphInstantiate(&c->iter_graph, graph, 0) == cudaSuccess;
+            if (graph) cudaGraphDestroy(graph);
+            c->iter_graph_launches = c->launches - before;
+            c->launches = before;                         // the captured iteration has not run
+            if (!ok) {
+                cudaGetLastError();
+                if (c->iter_graph) { cudaGraphExecDestroy(c->iter_graph); c->iter_graph = nullptr; }
+                c->iter_graph_off = true;
+            } else {
+                c->iter_graph_key = key;
+            }
+        }
+        if (c->iter_graph) {
+            for (; done < steps; ++done) {
+                CU(cudaGraphLaunch(c->iter_graph, c->stream));
+                c->launches += c->iter_graph_launches;
+            }
+        }
+    } else {
+        cudaGetLastError();
+    }
+    for (; done < steps; ++done) EF(enqueue_launch_iteration(c));
+    c->last_path = EF21_PATH_LAUNCHES;
+    return EF21_OK;
+}
+
 ef21_status ef21_step(ef21_ctx* c, int32_t steps) {
     if (!c || steps < 0) return EF21_ERR_INVALID_ARG;
     if (!c->shards_loaded || !c->inited) return EF21_ERR_STATE;
     if (steps == 0) return EF21_OK;
-    if (c->variant == EF21_VARIANT_EF) {
+    if (c->variant != EF21_VARIANT_EF21) {
         if (c->path == EF21_PATH_PERSISTENT) return EF21_ERR_UNSUPPORTED;
-        for (int t = 0; t < steps; ++t) {
-            EF(enqueue_grads(c, false));
-            EF(enqueue_ef_round(c, c->at<float>(c->L.grad), c->L.ld));
-        }
-        c->last_path = EF21_PATH_LAUNCHES;
-        return EF21_OK;
-    }
-    if (c->variant == EF21_VARIANT_EF21_PLUS) {
-        if (c->path == EF21_PATH_PERSISTENT) return EF21_ERR_UNSUPPORTED;
-        for (int t = 0; t < steps; ++t) {
-            EF(enqueue_x_update(c));
-            EF(enqueue_grads(c, false));
-            EF(enqueue_plus_round(c, c->at<float>(c->L.grad), c->L.ld));
-        }
-        c->last_path = EF21_PATH_LAUNCHES;
-        return EF21_OK;
+        return run_launch_iterations(c, steps);
     }
     if (c->path != EF21_PATH_LAUNCHES) {
         PersistPlan P = plan_persistent(c);
@@ -852,13 +911,7 @@ ef21_status ef21_step(ef21_ctx* c, int32_t steps) {
         }
         if (c->path == EF21_PATH_PERSISTENT) return EF21_ERR_UNSUPPORTED;
     }
-    for (int t = 0; t < steps; ++t) {
-        EF(enqueue_x_update(c));
-        EF(enqueue_grads(c, false));
-        EF(enqueue_round(c, c->at<float>(c->L.grad), c->L.ld, false));
-    }
-    c->last_path = EF21_PATH_LAUNCHES;
-    return EF21_OK;
+    return run_launch_iterations(c, steps);
 }
 
 ef21_status ef21_step_grads(ef21_ctx* c, const float* V_dev, int32_t steps) {

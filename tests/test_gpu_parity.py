@@ -146,6 +146,30 @@ def test_topk_short_vectors_one_launch(d, k, B, oracle32):
         np.testing.assert_array_equal(val[i].view(np.uint32), wv.view(np.uint32))
 
 
+@pytest.mark.parametrize("variant", [0, 1, 2])
+@pytest.mark.parametrize("side_stream", [False, True])
+def test_launch_path_many_steps_in_one_call_equal_single_steps(variant, side_stream, B):
+    # a call of several iterations replays the iteration as a graph from the second one on: same bits as
+    # one call per iteration, on the default stream and on a stream of the caller's, for every method
+    import torch
+    w = inputs.config(2, k=4)
+    outs = []
+    for chunks in ((12,), (1,) * 12, (5, 1, 6)):
+        stream = torch.cuda.Stream() if side_stream else None
+        with torch.cuda.stream(stream) if stream is not None else torch.cuda.stream(torch.cuda.current_stream()):
+            h = B.EF21(w.n, w.d, 4, w.gamma, w.lam, total_rows=w.N, stream=stream)
+            h.set_path(B.PATH_LAUNCHES); h.set_variant(variant)
+            h.load_shards(dev(w.A), dev(w.y), w.row_offsets)
+            h.init(B.INIT_ZERO if variant == 2 else B.INIT_COMPRESSED)
+            for s_ in chunks:
+                h.step(s_)
+            outs.append(h.get_state_host())
+            assert h.poll() == 0 and h.last_path == B.PATH_LAUNCHES
+    for other in outs[1:]:
+        for a_, b_ in zip(outs[0], other):
+            np.testing.assert_array_equal(a_, b_)
+
+
 def test_eval_matches_oracle(B, oracle32):
     w = inputs.config(0)
     h = make_gpu(w); h.init(B.INIT_COMPRESSED); h.step(5)
