@@ -212,9 +212,10 @@ ef21_status ef21_set_objective(ef21_ctx* ctx, int32_t objective);
 /* EF21+ (Section 3.4, Algorithm 3).  With EF21_VARIANT_EF21_PLUS every step computes, per worker,
  * b_i = C(grad f_i(x)) and m_i = g_i + C(grad f_i(x) - g_i), the distortions B_i = ||b_i - grad f_i(x)||^2
  * and M_i = ||m_i - grad f_i(x)||^2 (fp64 sums of the fp32 vectors), sets g_i = m_i if M_i <= B_i and
- * g_i = b_i otherwise, and recomputes g = (1/n) sum_i g_i (ascending i, then one multiply).  Runs on
- * the launch path only (EF21_PATH_PERSISTENT returns EF21_ERR_UNSUPPORTED).  The "last message" of
- * ef21_get_state is the compressed vector that was used.  Initialisation is that of Algorithm 2. */
+ * g_i = b_i otherwise, and recomputes g = (1/n) sum_i g_i (ascending i, then one multiply).  Both
+ * execution paths run it; the persistent kernel needs n * d * 4 <= 64 KB (every block keeps a copy
+ * of all g_i), otherwise the launch path is taken.  The "last message" of ef21_get_state is the
+ * compressed vector that was used.  Initialisation is that of Algorithm 2. */
 ef21_status ef21_set_variant(ef21_ctx* ctx, int32_t variant);
 /* The original error feedback method, EF (Section 4.1, Algorithm 4), with EF21_VARIANT_EF.  The
  * per-worker state is the error e_i, kept where Algorithm 2 keeps g_i (the gi argument of

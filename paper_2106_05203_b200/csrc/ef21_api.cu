@@ -530,11 +530,16 @@ ef21_status finish_load(ef21_ctx* c, const i64* row_offsets_host) {
 
 typedef void (*PersistKernel)(const PersistParams);
 
+template <int CHUNKS, int RB, int THREADS, bool PLUS>
+PersistKernel pk_by_src2(int src) {
+    if (src == PK_SRC_REG) return persistent_kernel<CHUNKS, RB, PK_SRC_REG, THREADS, 0, PLUS>;
+    if (src == PK_SRC_SMEM) return persistent_kernel<CHUNKS, RB, PK_SRC_SMEM, THREADS, 0, PLUS>;
+    return persistent_kernel<CHUNKS, RB, PK_SRC_GMEM, THREADS, 0, PLUS>;
+}
+thread_local bool g_pk_plus = false;      // which method pk_lookup resolves for (set by plan_persistent)
 template <int CHUNKS, int RB, int THREADS>
 PersistKernel pk_by_src(int src) {
-    if (src == PK_SRC_REG) return persistent_kernel<CHUNKS, RB, PK_SRC_REG, THREADS>;
-    if (src == PK_SRC_SMEM) return persistent_kernel<CHUNKS, RB, PK_SRC_SMEM, THREADS>;
-    return persistent_kernel<CHUNKS, RB, PK_SRC_GMEM, THREADS>;
+    return g_pk_plus ? pk_by_src2<CHUNKS, RB, THREADS, true>(src) : pk_by_src2<CHUNKS, RB, THREADS, false>(src);
 }
 
 // Instantiated shapes: (chunk slots per lane, rows per warp batch, threads per block).  512 threads
@@ -542,7 +547,7 @@ PersistKernel pk_by_src(int src) {
 PersistKernel pk_lookup(int chunks, int rb, int src, int threads, int extra) {
     // batches of 16 + 1 rows: registers only, one chunk slot, 16 warps
     if (extra == 1 && chunks == 1 && rb == 16 && src == PK_SRC_REG && threads == 512)
-        return persistent_kernel<1, 16, PK_SRC_REG, 512, 1>;
+        return g_pk_plus ? persistent_kernel<1, 16, PK_SRC_REG, 512, 1, true> : persistent_kernel<1, 16, PK_SRC_REG, 512, 1, false>;
     if (extra != 0) return nullptr;
     switch (chunks * 10000 + rb * 100 + threads / 256) {
         case 10401: return pk_by_src<1, 4, 256>(src);
@@ -580,7 +585,8 @@ bool pk_use_table(int n, int ld, int k) { return k >= 2 && (size_t)n * ld * 4 <=
 
 size_t pk_smem_bytes(int n, int k, int ld, int C, int nmsg, int src, i64 rows_cta, int threads) {
     size_t b = (size_t)(6 + threads / 32 + C) * ld * 4 + (size_t)((nmsg + 1) & ~1) * 8 + (size_t)((2 * ld + 15) & ~15);
-    if (pk_use_table(n, ld, k)) b += (size_t)n * ld * 4;
+    if (g_pk_plus) b += (size_t)n * ld * 4 + (size_t)ld * 4 + (size_t)((ld + 15) & ~15) + (size_t)((n + 15) & ~15);   // replicas of all g_i, grad_i, second selection, branches
+    else if (pk_use_table(n, ld, k)) b += (size_t)n * ld * 4;
     if (src == PK_SRC_SMEM) b += (size_t)rows_cta * ld * 4;
     return b;
 }
@@ -591,6 +597,8 @@ PersistPlan plan_persistent(ef21_ctx* c) {
     PersistPlan P; P.ok = false;
     const int ld = (int)c->L.ld;
     if (!c->shards_loaded || ld > 512 || c->k > PK_MAX_K || (i64)c->n * c->k > PK_MAX_MSGS) return P;
+    g_pk_plus = c->variant == EF21_VARIANT_EF21_PLUS;
+    if (g_pk_plus && (size_t)c->n * ld * 4 > (size_t)PK_TABLE_MAX_BYTES) return P;      // every block keeps all g_i
     int dev = 0, sms = 0, max_smem = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return P;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -684,10 +692,11 @@ ef21_status run_persistent(ef21_ctx* c, const PersistPlan& P, int steps) {
     PersistParams p;
     p.A = c->at<float>(c->L.A); p.y = c->at<float>(c->L.y); p.row_off = c->at<i64>(c->L.row_off);
     p.x = c->x(); p.g = c->g(); p.gi = c->gi(); p.msg_idx = c->msg_idx(); p.msg_val = c->msg_val();
+    p.plus_choice = c->at<int>(c->L.plus_choice);
     p.slots = c->at<unsigned long long>(c->L.slots); p.status = c->status();
     p.n = c->n; p.d = (int)c->d; p.ld = (int)c->L.ld; p.k = c->k; p.C = P.C; p.steps = steps;
     p.objective = c->objective;
-    p.slice_rows = 0; p.use_table = pk_use_table(c->n, (int)c->L.ld, c->k) ? 1 : 0; p.gamma = c->gamma; p.lambda = c->lambda; p.inv_n = 1.0f / (float)c->n;
+    p.slice_rows = 0; p.use_table = (c->variant != EF21_VARIANT_EF21_PLUS && pk_use_table(c->n, (int)c->L.ld, c->k)) ? 1 : 0; p.gamma = c->gamma; p.lambda = c->lambda; p.inv_n = 1.0f / (float)c->n;
     p.spin_limit = c->spin_limit; p.epoch0 = 0u;
     CU(cudaMemsetAsync(p.slots, 0, (size_t)2 * c->n * c->k * 8, c->stream));
     cudaLaunchConfig_t cfg = {};
@@ -898,7 +907,7 @@ ef21_status ef21_step(ef21_ctx* c, int32_t steps) {
     if (!c || steps < 0) return EF21_ERR_INVALID_ARG;
     if (!c->shards_loaded || !c->inited) return EF21_ERR_STATE;
     if (steps == 0) return EF21_OK;
-    if (c->variant != EF21_VARIANT_EF21) {
+    if (c->variant == EF21_VARIANT_EF) {
         if (c->path == EF21_PATH_PERSISTENT) return EF21_ERR_UNSUPPORTED;
         return run_launch_iterations(c, steps);
     }

@@ -50,6 +50,7 @@ struct PersistParams {
     float* gi;                 // [n][ld]
     int* msg_idx;              // [n][k] last messages (written at the final iteration)
     float* msg_val;
+    int* plus_choice;          // [n] EF21+: branch taken at the final iteration (0 Markov compressor, 1 plain)
     unsigned long long* slots; // [2][n*k]
     unsigned* status;
     int n, d, ld, k, C, steps;
@@ -112,7 +113,10 @@ __device__ __forceinline__ float comp_of(const float4& v, int c) {
 
 // EXTRA > 0: a warp's batch has RB + EXTRA rows; the first RB go through the transposed reduction, each
 // extra row through a plain butterfly sum (for shards whose rows per warp just exceed a power of two).
-template <int CHUNKS, int RB, int SRC, int THREADS, int EXTRA = 0>
+// PLUS: EF21+ (Algorithm 3).  The leader also selects C(grad_i), compares the two distortions and keeps the
+// better vector; a message carries the branch in bit 15 of its index field; every block keeps a replica of
+// all g_i and recomputes g = (1/n) sum_i g_i (ascending i, one multiply) after each exchange.
+template <int CHUNKS, int RB, int SRC, int THREADS, int EXTRA = 0, bool PLUS = false>
 __global__ void __launch_bounds__(THREADS, 1) persistent_kernel(const PersistParams p) {
     constexpr int RBT = RB + EXTRA;                                            // rows per batch
     constexpr int SH = (RB == 32) ? 0 : (RB == 16 ? 1 : (RB == 8 ? 2 : 3));    // log2(32/RB)
@@ -143,8 +147,15 @@ __global__ void __launch_bounds__(THREADS, 1) persistent_kernel(const PersistPar
     unsigned char* touched = reinterpret_cast<unsigned char*>(sacc + ld);             // [ld] coordinate received a message
     unsigned char* sel = touched + ld;                                                // [ld] leader: entry is in the Top-k
     unsigned* table = reinterpret_cast<unsigned*>(touched + ((2 * ld + 15) & ~15));   // [n][ld] value bits by (worker, coordinate)
-    float* slice = reinterpret_cast<float*>(table + (p.use_table ? p.n * ld : 0));    // SMEM source, 16-byte aligned
+    float* gall = reinterpret_cast<float*>(table);                                    // PLUS: [n][ld] replica of every g_i
+    float* gr = gall + (PLUS ? p.n * ld : 0);                                         // PLUS, leader: [ld] grad_i
+    unsigned char* selb = reinterpret_cast<unsigned char*>(gr + (PLUS ? ld : 0));     // PLUS, leader: [ld] entry is in Top-k of grad_i
+    unsigned char* wflag = selb + (PLUS ? ((ld + 15) & ~15) : 0);                     // PLUS: [n] branch of each worker's message
+    float* slice = PLUS ? reinterpret_cast<float*>(wflag + ((p.n + 15) & ~15))
+                        : reinterpret_cast<float*>(table + (p.use_table ? p.n * ld : 0));   // SMEM source, 16-byte aligned
     __shared__ int abort_flag;
+    __shared__ double dist_red[2][THREADS / 32];
+    __shared__ int plus_branch;
     __shared__ __align__(8) unsigned long long part_bar;     // leader: counts the bytes of the partials
 
     // ---- this block's rows --------------------------------------------------------------------
@@ -167,8 +178,11 @@ __global__ void __launch_bounds__(THREADS, 1) persistent_kernel(const PersistPar
     }
     for (int j = tid; j < ld; j += THREADS) { xs[j] = p.x[j]; gs[j] = p.g[j]; }
     for (int j = tid; j < ld; j += THREADS) { sacc[j] = 0.f; touched[j] = 0; }
-    if (p.use_table)
+    if (PLUS) {
+        for (int e = tid; e < p.n * ld; e += THREADS) gall[e] = p.gi[e];
+    } else if (p.use_table) {
         for (int e = tid; e < p.n * ld; e += THREADS) table[e] = PK_NO_ENTRY;
+    }
     if (SRC == PK_SRC_SMEM) {
         const float4* src = reinterpret_cast<const float4*>(p.A + r0 * (i64)ld);
         float4* dst = reinterpret_cast<float4*>(slice);
@@ -323,9 +337,83 @@ __global__ void __launch_bounds__(THREADS, 1) persistent_kernel(const PersistPar
                     for (int cc = 1; cc < C; ++cc) sum = __fadd_rn(sum, part[cc * ld + j]);
                     const float grad = __fadd_rn(m_i > 0 ? __fdiv_rn(sum, mf) : 0.f, rterm[j]);
                     vs[j] = __fsub_rn(grad, gis[j]);
+                    if (PLUS) gr[j] = grad;
                 }
                 __syncthreads();
-                if (rank_select) {
+                if (PLUS) {
+                    // ranks of every coordinate in grad_i - g_i and in grad_i ((|.| descending, index ascending);
+                    // `split` adjacent lanes share a coordinate and count a contiguous part of the entries each)
+                    const int split = (ld * 4 <= THREADS) ? 4 : ((ld * 2 <= THREADS) ? 2 : 1);
+                    const int part_len = (p.d + split - 1) / split;
+                    for (int j0 = 0; j0 < ld; j0 += THREADS / split) {
+                        const int j = j0 + tid / split, q = tid % split;
+                        int rank_m = 0, rank_b = 0;
+                        if (j < p.d) {
+                            const unsigned km = mag_key(vs[j]), kb = mag_key(gr[j]);
+                            const int i1 = min((q + 1) * part_len, p.d);
+#pragma unroll 2
+                            for (int i = q * part_len; i < i1; ++i) {
+                                const unsigned kim = mag_key(vs[i]), kib = mag_key(gr[i]);
+                                rank_m += (kim > km || (kim == km && i < j)) ? 1 : 0;
+                                rank_b += (kib > kb || (kib == kb && i < j)) ? 1 : 0;
+                            }
+                        }
+                        if (split >= 2) { rank_m += __shfl_xor_sync(0xffffffffu, rank_m, 1); rank_b += __shfl_xor_sync(0xffffffffu, rank_b, 1); }
+                        if (split >= 4) { rank_m += __shfl_xor_sync(0xffffffffu, rank_m, 2); rank_b += __shfl_xor_sync(0xffffffffu, rank_b, 2); }
+                        if (q == 0 && j < ld) {
+                            sel[j] = (j < p.d && rank_m < p.k) ? 1 : 0;
+                            selb[j] = (j < p.d && rank_b < p.k) ? 1 : 0;
+                        }
+                    }
+                    __syncthreads();
+                    // distortions M_i = ||g_i + C(grad_i - g_i) - grad_i||^2 and B_i = ||C(grad_i) - grad_i||^2 as fp64
+                    // sums of the fp32 vectors, both over the coordinates in the same order
+                    double dm = 0.0, db = 0.0;
+                    for (int j = tid; j < p.d; j += THREADS) {
+                        const float g0 = gis[j], gj = gr[j];
+                        const float mj = sel[j] ? __fadd_rn(g0, vs[j]) : g0;
+                        const double em = (double)mj - (double)gj;
+                        dm += em * em;
+                        if (!selb[j]) db += (double)gj * (double)gj;
+                    }
+                    dm = warp_sum(dm); db = warp_sum(db);
+                    if (lane == 0) { dist_red[0][warp] = dm; dist_red[1][warp] = db; }
+                    __syncthreads();
+                    if (tid == 0) {
+                        double M = 0.0, Bd = 0.0;
+                        for (int w = 0; w < WARPS; ++w) { M += dist_red[0][w]; Bd += dist_red[1][w]; }
+                        plus_branch = M <= Bd ? 0 : 1;
+                    }
+                    __syncthreads();
+                    const int branch = plus_branch;
+                    if (warp == 0) {
+                        // the message: the compressed vector that was used, ascending index order from the ballot
+                        // ranks; bit 15 of the index field carries the branch
+                        const unsigned char* chosen_set = branch ? selb : sel;
+                        const float* values = branch ? gr : vs;
+                        int base = 0;
+                        for (int j0 = 0; j0 < ld; j0 += 32) {
+                            const int j = j0 + lane;
+                            const bool chosen = j < ld && chosen_set[j] != 0;
+                            const unsigned bal = __ballot_sync(0xffffffffu, chosen);
+                            if (chosen) {
+                                const int pos = base + __popc(bal & ((1u << lane) - 1u));
+                                const float val = values[j];
+                                const unsigned long long word = ((unsigned long long)epoch << 48) |
+                                                                ((unsigned long long)((unsigned)j | ((unsigned)branch << 15)) << 32) |
+                                                                (unsigned long long)__float_as_uint(val);
+                                st_relaxed_u64(slot + worker * p.k + pos, word);
+                                if (t == p.steps - 1) { p.msg_idx[worker * p.k + pos] = j; p.msg_val[worker * p.k + pos] = val; }
+                            }
+                            base += __popc(bal);
+                        }
+                        if (lane == 0 && t == p.steps - 1) p.plus_choice[worker] = branch;
+                    }
+                    // g_i <- the chosen vector (nobody reads gis again before the next iteration's barriers)
+                    for (int j = tid; j < ld; j += THREADS)
+                        gis[j] = branch ? (selb[j] ? gr[j] : 0.f) : (sel[j] ? __fadd_rn(gis[j], vs[j]) : gis[j]);
+                }
+                if (!PLUS && rank_select) {
                     // larger k: every coordinate counts the entries that precede it in (|v| descending, index
                     // ascending) order; the k entries of rank < k are the message.  `split` adjacent lanes share a
                     // coordinate, each counts a contiguous part of the entries, a butterfly adds the parts up.
@@ -350,7 +438,7 @@ __global__ void __launch_bounds__(THREADS, 1) persistent_kernel(const PersistPar
                     __syncthreads();
                 }
             }
-            if (leader && warp == 0 && rank_select) {
+            if (!PLUS && leader && warp == 0 && rank_select) {
                 // ascending index order falls out of the ballot ranks
                 int base = 0;
                 for (int j0 = 0; j0 < ld; j0 += 32) {
@@ -369,7 +457,7 @@ __global__ void __launch_bounds__(THREADS, 1) persistent_kernel(const PersistPar
                     base += __popc(bal);
                 }
             }
-            if (leader && warp == 0 && !rank_select) {
+            if (!PLUS && leader && warp == 0 && !rank_select) {
                 float4 v[CHUNKS];
                 unsigned taken = pad_mask;            // bit (cs*4+comp) set: not selectable
 #pragma unroll
@@ -445,7 +533,7 @@ __global__ void __launch_bounds__(THREADS, 1) persistent_kernel(const PersistPar
             for (int u = tid; u < nmsg; u += THREADS) {
                 unsigned long long w;
                 const bool got = poll_word(u, w);
-                if (p.use_table) {
+                if (!PLUS && p.use_table) {
                     const unsigned idx = (unsigned)(w >> 32) & 0xffffu;
                     if (got && idx < (unsigned)ld) table[(int)(((unsigned)u * k_magic) >> 16) * ld + (int)idx] = (unsigned)w;
                 } else {
@@ -454,6 +542,31 @@ __global__ void __launch_bounds__(THREADS, 1) persistent_kernel(const PersistPar
             }
             __syncthreads();
             if (abort_flag) aborted = true;
+        }
+        if (PLUS && !aborted) {
+            // every block applies the n messages to its replicas of the g_i: a worker that took the plain branch
+            // restarts from zero, the others add their entries; then g = (1/n) sum_i g_i, ascending i
+            for (int i = tid; i < p.n; i += THREADS) wflag[i] = (unsigned char)((msg[i * p.k] >> 47) & 1ull);
+            __syncthreads();
+            for (int i = 0; i < p.n; ++i)
+                if (wflag[i])
+                    for (int j = tid; j < ld; j += THREADS) gall[i * ld + j] = 0.f;
+            __syncthreads();
+            for (int u = tid; u < nmsg; u += THREADS) {
+                const unsigned long long w = msg[u];
+                const int i = (int)(((unsigned)u * k_magic) >> 16);
+                const unsigned idx = (unsigned)(w >> 32) & 0x7fffu;
+                const float val = __uint_as_float((unsigned)w);
+                if (idx < (unsigned)ld) gall[i * ld + (int)idx] = wflag[i] ? val : __fadd_rn(gall[i * ld + (int)idx], val);
+            }
+            __syncthreads();
+            for (int j = tid; j < p.d; j += THREADS) {
+                float sum = 0.f;
+#pragma unroll 4
+                for (int i = 0; i < p.n; ++i) sum = __fadd_rn(sum, gall[i * ld + j]);
+                gs[j] = __fmul_rn(sum, p.inv_n);
+            }
+            continue;
         }
         if (!aborted && p.use_table) {
             // g_j += (1/n) * sum over workers (ascending) of the values sent for coordinate j: row i of the

@@ -64,32 +64,61 @@ def test_supplied_gradients_both_branches_bit_exact(n, d, k, B, oracle32):
     assert h.poll() == 0
 
 
-def test_logistic_ef21_plus_tracks_the_oracle(B, oracle32):
-    w = inputs.config(0)
-    h = make_gpu(w); h.set_variant(B.VARIANT_EF21_PLUS)
-    st = make_oracle_state(oracle32, w)
+@pytest.mark.parametrize("path", [1, 2])
+@pytest.mark.parametrize("cfg,k", [(0, 4), (1, 1), (2, 16)])
+def test_logistic_ef21_plus_tracks_the_oracle(cfg, k, path, B, oracle32):
+    # launch-per-stage kernels (path 1) and the persistent cluster kernel (path 2)
+    w = inputs.config(cfg, k=k)
+    h = make_gpu(w, k=k, path=path); h.set_variant(B.VARIANT_EF21_PLUS)
+    st = make_oracle_state(oracle32, w, k=k)
     h.init(0); st.init(0)
+    rebased = 0
     for t in range(30):
+        gi_old = st.gi.copy()
         h.step(1); st.plus_step(1)
+        assert h.last_path == path
         x, g, gi, li, lv = h.get_state_host()
-        np.testing.assert_array_equal(h.get_plus_choice(), st.choice)
-        np.testing.assert_array_equal(li, st.idx)
-        assert rel_l2(x, st.x) <= 1e-4 or np.linalg.norm(st.x) == 0
-        assert np.max(np.abs(gi - st.gi)) <= 1e-5 * np.max(np.abs(st.gi))
+        if not (np.array_equal(h.get_plus_choice(), st.choice) and np.array_equal(li, st.idx)):
+            # only a near-tie (between two entries, or between the two distortions) may change a decision
+            grads = st.grads().astype(np.float64)
+            for i in range(w.n):
+                if h.get_plus_choice()[i] != st.choice[i]:
+                    continue            # distortions within rounding of each other; checked by the bound on rebasings
+                v = grads[i] - gi_old[i] if st.choice[i] == 0 else grads[i]
+                kth = np.sort(np.abs(v))[::-1][k - 1]
+                for j in set(li[i].tolist()) ^ set(st.idx[i].tolist()):
+                    assert abs(abs(v[j]) - kth) <= 4e-5 * (np.max(np.abs(grads[i])) + 1e-30), (t, i, j)
+            rebased += 1
+        else:
+            assert rel_l2(x, st.x) <= 1e-4 or np.linalg.norm(st.x) == 0
+            assert np.max(np.abs(gi - st.gi)) <= 1e-5 * np.max(np.abs(st.gi))
+            assert np.max(np.abs(g - st.g)) <= 1e-5 * np.max(np.abs(st.gi))      # g is a mean of the g_i: their scale
         set_gpu_state_from_oracle(h, st)
-    assert h.last_path == B.PATH_LAUNCHES
-    h.set_path(B.PATH_PERSISTENT)
-    with pytest.raises(B.Ef21Error) as e:
-        h.step(1)
-    assert e.value.status == 7
+    assert rebased <= 3
+    assert h.poll() == 0
 
 
-def test_free_running_ef21_plus_paper_shape(B, oracle32):
+@pytest.mark.parametrize("path", [1, 2])
+def test_free_running_ef21_plus_paper_shape(path, B, oracle32):
     w = inputs.config(1)
-    h = make_gpu(w); h.set_variant(B.VARIANT_EF21_PLUS)
+    h = make_gpu(w, path=path); h.set_variant(B.VARIANT_EF21_PLUS)
     st = make_oracle_state(oracle32, w)
     h.init(0); st.init(0)
     h.step(60); st.plus_step(60)
+    assert h.last_path == path
     x = h.get_state_host()[0]
     assert rel_l2(x, st.x) <= 1e-4
     assert h.eval()[0] == pytest.approx(st.loss(), rel=1e-4)
+
+
+def test_persistent_ef21_plus_many_steps_in_one_launch_equal_single_steps(B):
+    w = inputs.config(2, k=4)
+    outs = []
+    for chunks in ((12,), (1,) * 12):
+        h = make_gpu(w, k=4, path=2); h.set_variant(B.VARIANT_EF21_PLUS)
+        h.init(0)
+        for s_ in chunks:
+            h.step(s_)
+        outs.append(h.get_state_host() + (h.get_plus_choice(),))
+    for a_, b_ in zip(outs[0], outs[1]):
+        np.testing.assert_array_equal(a_, b_)
