@@ -532,9 +532,14 @@ typedef void (*PersistKernel)(const PersistParams);
 
 template <int CHUNKS, int RB, int THREADS, bool PLUS>
 PersistKernel pk_by_src2(int src) {
-    if (src == PK_SRC_REG) return persistent_kernel<CHUNKS, RB, PK_SRC_REG, THREADS, 0, PLUS>;
-    if (src == PK_SRC_SMEM) return persistent_kernel<CHUNKS, RB, PK_SRC_SMEM, THREADS, 0, PLUS>;
-    return persistent_kernel<CHUNKS, RB, PK_SRC_GMEM, THREADS, 0, PLUS>;
+    if (PLUS) {
+        if (src == PK_SRC_REG) return persistent_plus_kernel<CHUNKS, RB, PK_SRC_REG, THREADS, 0>;
+        if (src == PK_SRC_SMEM) return persistent_plus_kernel<CHUNKS, RB, PK_SRC_SMEM, THREADS, 0>;
+        return persistent_plus_kernel<CHUNKS, RB, PK_SRC_GMEM, THREADS, 0>;
+    }
+    if (src == PK_SRC_REG) return persistent_kernel<CHUNKS, RB, PK_SRC_REG, THREADS, 0>;
+    if (src == PK_SRC_SMEM) return persistent_kernel<CHUNKS, RB, PK_SRC_SMEM, THREADS, 0>;
+    return persistent_kernel<CHUNKS, RB, PK_SRC_GMEM, THREADS, 0>;
 }
 thread_local bool g_pk_plus = false;      // which method pk_lookup resolves for (set by plan_persistent)
 template <int CHUNKS, int RB, int THREADS>
@@ -547,7 +552,7 @@ PersistKernel pk_by_src(int src) {
 PersistKernel pk_lookup(int chunks, int rb, int src, int threads, int extra) {
     // batches of 16 + 1 rows: registers only, one chunk slot, 16 warps
     if (extra == 1 && chunks == 1 && rb == 16 && src == PK_SRC_REG && threads == 512)
-        return g_pk_plus ? persistent_kernel<1, 16, PK_SRC_REG, 512, 1, true> : persistent_kernel<1, 16, PK_SRC_REG, 512, 1, false>;
+        return g_pk_plus ? persistent_plus_kernel<1, 16, PK_SRC_REG, 512, 1> : persistent_kernel<1, 16, PK_SRC_REG, 512, 1>;
     if (extra != 0) return nullptr;
     switch (chunks * 10000 + rb * 100 + threads / 256) {
         case 10401: return pk_by_src<1, 4, 256>(src);
@@ -585,7 +590,7 @@ bool pk_use_table(int n, int ld, int k) { return k >= 2 && (size_t)n * ld * 4 <=
 
 size_t pk_smem_bytes(int n, int k, int ld, int C, int nmsg, int src, i64 rows_cta, int threads) {
     size_t b = (size_t)(6 + threads / 32 + C) * ld * 4 + (size_t)((nmsg + 1) & ~1) * 8 + (size_t)((2 * ld + 15) & ~15);
-    if (g_pk_plus) b += (size_t)n * ld * 4 + (size_t)ld * 4 + (size_t)((ld + 15) & ~15) + (size_t)((n + 15) & ~15);   // replicas of all g_i, grad_i, second selection, branches
+    if (g_pk_plus) b += (size_t)n * ld * 4 + (size_t)ld * 4 + (size_t)((ld + 15) & ~15) + (size_t)((n + 15) & ~15) + (size_t)2 * (threads / 32) * 8 + 16;   // replicas of all g_i, grad_i, second selection, branches, distortion partials
     else if (pk_use_table(n, ld, k)) b += (size_t)n * ld * 4;
     if (src == PK_SRC_SMEM) b += (size_t)rows_cta * ld * 4;
     return b;
