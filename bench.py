@@ -249,7 +249,7 @@ def run_ours(args):
         if variant == 0:
             h.set_path({"auto": B.PATH_AUTO, "launches": B.PATH_LAUNCHES, "persistent": B.PATH_PERSISTENT}[args.path])
         h.load_shards(dev(w.A), dev(w.y), w.row_offsets)
-        h.init(B.INIT_COMPRESSED)
+        h.init(B.INIT_ZERO if variant == B.VARIANT_EF else B.INIT_COMPRESSED)      # Algorithm 4 starts from e_i = 0
         x0, g0, gi0, _, _ = h.get_state()
         h.step(warmup)
         times, launches = [], 0
@@ -381,11 +381,15 @@ def run_ours(args):
                            "launches": rr["launches"], "persistent_shape": rr["shape"], "f_end": rr["f_end"]})
         others.append(time_stress(None, 50, 3))
         others.append(time_hbm_scale(50, 3))
-        # EF21+ (Algorithm 3) on the headline shapes: launch-per-stage kernels, two Top-k per worker and step
+        # EF21+ (Algorithm 3) on the headline shapes (persistent_plus_kernel)
         wp = inputs.config(HEADLINE)
         rp = time_logistic(wp, wp.k, 500, 10, variant=B.VARIANT_EF21_PLUS)
         others.append({"workload": f"EF21+ on configs[{HEADLINE}] {wp.name} Top-{wp.k}", "iterations_per_s": 500 / (rp["ms"] * 1e-3),
                        "us_per_iteration": rp["ms"] / 500 * 1e3, "launches": rp["launches"], "f_end": rp["f_end"]})
+        # EF, the original error feedback method (Algorithm 4), same shapes
+        re_ = time_logistic(wp, wp.k, 500, 10, variant=B.VARIANT_EF)
+        others.append({"workload": f"EF (Algorithm 4) on configs[{HEADLINE}] {wp.name} Top-{wp.k}", "iterations_per_s": 500 / (re_["ms"] * 1e-3),
+                       "us_per_iteration": re_["ms"] / 500 * 1e3, "launches": re_["launches"], "f_end": re_["f_end"]})
         line["workloads"] = others
 
     if world > 1:

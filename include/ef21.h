@@ -228,7 +228,8 @@ ef21_status ef21_set_variant(ef21_ctx* ctx, int32_t variant);
  * and e_i^{t+1}.  The "last message" of ef21_get_state is w_i^{t-1}.  gamma * grad, the sum with
  * e_i, the difference with w_i, the factor 1/n and the update of x are single rounded fp32
  * operations; the sum over workers runs in ascending worker order.  ef21_step_grads uses the
- * supplied vectors in place of grad f_i.  Launch path only; ef21_step_minibatch is not available. */
+ * supplied vectors in place of grad f_i.  Both execution paths run ef21_step; ef21_step_minibatch
+ * is not available. */
 /* choice_host[n]: 0 where the last EF21+ step kept the Markov compressor, 1 where it took C(grad);
  * synchronises. */
 ef21_status ef21_get_plus_choice(ef21_ctx* ctx, int32_t* choice_host);

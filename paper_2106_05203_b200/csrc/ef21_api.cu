@@ -530,9 +530,14 @@ ef21_status finish_load(ef21_ctx* c, const i64* row_offsets_host) {
 
 typedef void (*PersistKernel)(const PersistParams);
 
-template <int CHUNKS, int RB, int THREADS, bool PLUS>
+template <int CHUNKS, int RB, int THREADS, int METHOD>
 PersistKernel pk_by_src2(int src) {
-    if (PLUS) {
+    if (METHOD == EF21_VARIANT_EF) {
+        if (src == PK_SRC_REG) return persistent_ef_kernel<CHUNKS, RB, PK_SRC_REG, THREADS, 0>;
+        if (src == PK_SRC_SMEM) return persistent_ef_kernel<CHUNKS, RB, PK_SRC_SMEM, THREADS, 0>;
+        return persistent_ef_kernel<CHUNKS, RB, PK_SRC_GMEM, THREADS, 0>;
+    }
+    if (METHOD == EF21_VARIANT_EF21_PLUS) {
         if (src == PK_SRC_REG) return persistent_plus_kernel<CHUNKS, RB, PK_SRC_REG, THREADS, 0>;
         if (src == PK_SRC_SMEM) return persistent_plus_kernel<CHUNKS, RB, PK_SRC_SMEM, THREADS, 0>;
         return persistent_plus_kernel<CHUNKS, RB, PK_SRC_GMEM, THREADS, 0>;
@@ -542,9 +547,11 @@ PersistKernel pk_by_src2(int src) {
     return persistent_kernel<CHUNKS, RB, PK_SRC_GMEM, THREADS, 0>;
 }
 thread_local bool g_pk_plus = false;      // which method pk_lookup resolves for (set by plan_persistent)
+thread_local bool g_pk_ef = false;
 template <int CHUNKS, int RB, int THREADS>
 PersistKernel pk_by_src(int src) {
-    return g_pk_plus ? pk_by_src2<CHUNKS, RB, THREADS, true>(src) : pk_by_src2<CHUNKS, RB, THREADS, false>(src);
+    if (g_pk_ef) return pk_by_src2<CHUNKS, RB, THREADS, EF21_VARIANT_EF>(src);
+    return g_pk_plus ? pk_by_src2<CHUNKS, RB, THREADS, EF21_VARIANT_EF21_PLUS>(src) : pk_by_src2<CHUNKS, RB, THREADS, EF21_VARIANT_EF21>(src);
 }
 
 // Instantiated shapes: (chunk slots per lane, rows per warp batch, threads per block).  512 threads
@@ -552,7 +559,8 @@ PersistKernel pk_by_src(int src) {
 PersistKernel pk_lookup(int chunks, int rb, int src, int threads, int extra) {
     // batches of 16 + 1 rows: registers only, one chunk slot, 16 warps
     if (extra == 1 && chunks == 1 && rb == 16 && src == PK_SRC_REG && threads == 512)
-        return g_pk_plus ? persistent_plus_kernel<1, 16, PK_SRC_REG, 512, 1> : persistent_kernel<1, 16, PK_SRC_REG, 512, 1>;
+        return g_pk_ef ? persistent_ef_kernel<1, 16, PK_SRC_REG, 512, 1>
+                       : (g_pk_plus ? persistent_plus_kernel<1, 16, PK_SRC_REG, 512, 1> : persistent_kernel<1, 16, PK_SRC_REG, 512, 1>);
     if (extra != 0) return nullptr;
     switch (chunks * 10000 + rb * 100 + threads / 256) {
         case 10401: return pk_by_src<1, 4, 256>(src);
@@ -603,6 +611,7 @@ PersistPlan plan_persistent(ef21_ctx* c) {
     const int ld = (int)c->L.ld;
     if (!c->shards_loaded || ld > 512 || c->k > PK_MAX_K || (i64)c->n * c->k > PK_MAX_MSGS) return P;
     g_pk_plus = c->variant == EF21_VARIANT_EF21_PLUS;
+    g_pk_ef = c->variant == EF21_VARIANT_EF;
     if (g_pk_plus && (size_t)c->n * ld * 4 > (size_t)PK_TABLE_MAX_BYTES) return P;      // every block keeps all g_i
     int dev = 0, sms = 0, max_smem = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return P;
@@ -912,10 +921,6 @@ ef21_status ef21_step(ef21_ctx* c, int32_t steps) {
     if (!c || steps < 0) return EF21_ERR_INVALID_ARG;
     if (!c->shards_loaded || !c->inited) return EF21_ERR_STATE;
     if (steps == 0) return EF21_OK;
-    if (c->variant == EF21_VARIANT_EF) {
-        if (c->path == EF21_PATH_PERSISTENT) return EF21_ERR_UNSUPPORTED;
-        return run_launch_iterations(c, steps);
-    }
     if (c->path != EF21_PATH_LAUNCHES) {
         PersistPlan P = plan_persistent(c);
         if (P.ok) {

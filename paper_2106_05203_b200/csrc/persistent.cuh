@@ -112,6 +112,7 @@ __device__ __forceinline__ float comp_of(const float4& v, int c) {
 }
 #define PK_KERNEL_NAME persistent_kernel
 #define PK_PLUS 0
+#define PK_EF 0
 #include "persistent_body.inc"
 #undef PK_KERNEL_NAME
 #undef PK_PLUS
@@ -120,6 +121,14 @@ __device__ __forceinline__ float comp_of(const float4& v, int c) {
 #include "persistent_body.inc"
 #undef PK_KERNEL_NAME
 #undef PK_PLUS
+#undef PK_EF
+#define PK_KERNEL_NAME persistent_ef_kernel
+#define PK_PLUS 0
+#define PK_EF 1
+#include "persistent_body.inc"
+#undef PK_KERNEL_NAME
+#undef PK_PLUS
+#undef PK_EF
 
 // One-block self-check of the bounded wait: spins on a word that nobody writes and must come back
 // with EF21_ERR_TIMEOUT in the status word instead of hanging.

@@ -80,11 +80,14 @@ def test_supplied_gradients_multi_step_call_equals_single_steps(B):
     np.testing.assert_array_equal(outs[0][1].view(np.uint32), outs[1][1].view(np.uint32))
 
 
-def test_logistic_ef_tracks_the_oracle(B, oracle32, oracle64):
-    w = inputs.config(0)
-    h = make_gpu(w); h.set_variant(B.VARIANT_EF)
+@pytest.mark.parametrize("path", [1, 2])
+@pytest.mark.parametrize("cfg,k", [(0, 4), (1, 1), (2, 16)])
+def test_logistic_ef_tracks_the_oracle(cfg, k, path, B, oracle32, oracle64):
+    # launch-per-stage kernels (path 1) and the persistent cluster kernel (path 2)
+    w = inputs.config(cfg, k=k)
+    h = make_gpu(w, k=k, path=path); h.set_variant(B.VARIANT_EF)
     h.init(B.INIT_ZERO)
-    st = _ef_oracle(oracle32, w)
+    st = _ef_oracle(oracle32, w, k=k)
     st.init()
     rebased = 0
     for t in range(40):
@@ -106,30 +109,41 @@ def test_logistic_ef_tracks_the_oracle(B, oracle32, oracle64):
         assert np.max(np.abs(e - st.e)) <= 1e-5 * max(np.max(np.abs(st.e)), w.gamma * 1.0)
         h.set_state(dev(st.x), None, dev(st.e))
     assert rebased <= 4
-    assert h.last_path == B.PATH_LAUNCHES and h.poll() == 0
+    assert h.last_path == path and h.poll() == 0
 
 
-def test_free_running_ef_paper_shape(B, oracle32):
+@pytest.mark.parametrize("path", [1, 2])
+def test_free_running_ef_paper_shape(path, B, oracle32):
     w = inputs.config(1)
-    h = make_gpu(w); h.set_variant(B.VARIANT_EF)
+    h = make_gpu(w, path=path); h.set_variant(B.VARIANT_EF)
     h.init(B.INIT_ZERO)
     st = _ef_oracle(oracle32, w)
     st.init()
     h.step(60); st.step(60)
+    assert h.last_path == path
     x = h.get_state_host()[0]
     assert rel_l2(x, st.x) <= 1e-4
     assert h.eval()[0] == pytest.approx(st.loss(), rel=1e-4)
 
 
-def test_ef_is_launch_path_only(B):
+def test_persistent_ef_many_steps_in_one_launch_equal_single_steps(B):
+    w = inputs.config(2, k=4)
+    outs = []
+    for chunks in ((12,), (1,) * 12):
+        h = make_gpu(w, k=4, path=2); h.set_variant(B.VARIANT_EF)
+        h.init(B.INIT_ZERO)
+        for s_ in chunks:
+            h.step(s_)
+        assert h.last_path == 2
+        outs.append(h.get_state_host())
+    for a_, b_ in zip(outs[0], outs[1]):
+        np.testing.assert_array_equal(a_, b_)
+
+
+def test_ef_has_no_minibatch_step(B):
     w = inputs.config(0)
     h = make_gpu(w); h.set_variant(B.VARIANT_EF)
     h.init(B.INIT_ZERO)
-    h.set_path(B.PATH_PERSISTENT)
-    with pytest.raises(B.Ef21Error) as e:
-        h.step(1)
-    assert e.value.status == 7
-    h.set_path(B.PATH_AUTO)
     batch = dev(inputs.minibatch_rows(0, 0, w.row_offsets, 8), dtype=torch.int32)
     with pytest.raises(B.Ef21Error) as e:
         h.step_minibatch(batch)
