@@ -13,6 +13,7 @@
 #include "ef.cuh"
 #include "grad.cuh"
 #include "persistent.cuh"
+#include "wait_selftest.cuh"
 #include "plus.cuh"
 #include "stress.cuh"
 #include "topk.cuh"
@@ -528,63 +529,6 @@ ef21_status finish_load(ef21_ctx* c, const i64* row_offsets_host) {
 // Persistent path
 // ---------------------------------------------------------------------------------------------
 
-typedef void (*PersistKernel)(const PersistParams);
-
-template <int CHUNKS, int RB, int THREADS, int METHOD>
-PersistKernel pk_by_src2(int src) {
-    if (METHOD == EF21_VARIANT_EF) {
-        if (src == PK_SRC_REG) return persistent_ef_kernel<CHUNKS, RB, PK_SRC_REG, THREADS, 0>;
-        if (src == PK_SRC_SMEM) return persistent_ef_kernel<CHUNKS, RB, PK_SRC_SMEM, THREADS, 0>;
-        return persistent_ef_kernel<CHUNKS, RB, PK_SRC_GMEM, THREADS, 0>;
-    }
-    if (METHOD == EF21_VARIANT_EF21_PLUS) {
-        if (src == PK_SRC_REG) return persistent_plus_kernel<CHUNKS, RB, PK_SRC_REG, THREADS, 0>;
-        if (src == PK_SRC_SMEM) return persistent_plus_kernel<CHUNKS, RB, PK_SRC_SMEM, THREADS, 0>;
-        return persistent_plus_kernel<CHUNKS, RB, PK_SRC_GMEM, THREADS, 0>;
-    }
-    if (src == PK_SRC_REG) return persistent_kernel<CHUNKS, RB, PK_SRC_REG, THREADS, 0>;
-    if (src == PK_SRC_SMEM) return persistent_kernel<CHUNKS, RB, PK_SRC_SMEM, THREADS, 0>;
-    return persistent_kernel<CHUNKS, RB, PK_SRC_GMEM, THREADS, 0>;
-}
-thread_local bool g_pk_plus = false;      // which method pk_lookup resolves for (set by plan_persistent)
-thread_local bool g_pk_ef = false;
-template <int CHUNKS, int RB, int THREADS>
-PersistKernel pk_by_src(int src) {
-    if (g_pk_ef) return pk_by_src2<CHUNKS, RB, THREADS, EF21_VARIANT_EF>(src);
-    return g_pk_plus ? pk_by_src2<CHUNKS, RB, THREADS, EF21_VARIANT_EF21_PLUS>(src) : pk_by_src2<CHUNKS, RB, THREADS, EF21_VARIANT_EF21>(src);
-}
-
-// Instantiated shapes: (chunk slots per lane, rows per warp batch, threads per block).  512 threads
-// leave 128 registers per thread, so they exist only where a batch needs at most 16 float4 registers.
-PersistKernel pk_lookup(int chunks, int rb, int src, int threads, int extra) {
-    // batches of 16 + 1 rows: registers only, one chunk slot, 16 warps
-    if (extra == 1 && chunks == 1 && rb == 16 && src == PK_SRC_REG && threads == 512)
-        return g_pk_ef ? persistent_ef_kernel<1, 16, PK_SRC_REG, 512, 1>
-                       : (g_pk_plus ? persistent_plus_kernel<1, 16, PK_SRC_REG, 512, 1> : persistent_kernel<1, 16, PK_SRC_REG, 512, 1>);
-    if (extra != 0) return nullptr;
-    switch (chunks * 10000 + rb * 100 + threads / 256) {
-        case 10401: return pk_by_src<1, 4, 256>(src);
-        case 10801: return pk_by_src<1, 8, 256>(src);
-        case 11601: return pk_by_src<1, 16, 256>(src);
-        case 13201: return pk_by_src<1, 32, 256>(src);
-        case 20401: return pk_by_src<2, 4, 256>(src);
-        case 20801: return pk_by_src<2, 8, 256>(src);
-        case 21601: return pk_by_src<2, 16, 256>(src);
-        case 30401: return pk_by_src<3, 4, 256>(src);
-        case 30801: return pk_by_src<3, 8, 256>(src);
-        case 40401: return pk_by_src<4, 4, 256>(src);
-        case 40801: return pk_by_src<4, 8, 256>(src);
-        case 10402: return pk_by_src<1, 4, 512>(src);
-        case 10802: return pk_by_src<1, 8, 512>(src);
-        case 11602: return pk_by_src<1, 16, 512>(src);
-        case 20402: return pk_by_src<2, 4, 512>(src);
-        case 20802: return pk_by_src<2, 8, 512>(src);
-        case 30402: return pk_by_src<3, 4, 512>(src);
-        case 40402: return pk_by_src<4, 4, 512>(src);
-    }
-    return nullptr;
-}
-
 struct PersistPlan {
     bool ok;
     int C, rb, src, chunks, threads, extra;
@@ -596,9 +540,9 @@ struct PersistPlan {
 // memory (if that table is small): aggregation then costs n reads per coordinate instead of n*k.
 bool pk_use_table(int n, int ld, int k) { return k >= 2 && (size_t)n * ld * 4 <= (size_t)PK_TABLE_MAX_BYTES; }
 
-size_t pk_smem_bytes(int n, int k, int ld, int C, int nmsg, int src, i64 rows_cta, int threads) {
+size_t pk_smem_bytes(bool plus, int n, int k, int ld, int C, int nmsg, int src, i64 rows_cta, int threads) {
     size_t b = (size_t)(6 + threads / 32 + C) * ld * 4 + (size_t)((nmsg + 1) & ~1) * 8 + (size_t)((2 * ld + 15) & ~15);
-    if (g_pk_plus) b += (size_t)n * ld * 4 + (size_t)ld * 4 + (size_t)((ld + 15) & ~15) + (size_t)((n + 15) & ~15) + (size_t)2 * (threads / 32) * 8 + 16;   // replicas of all g_i, grad_i, second selection, branches, distortion partials
+    if (plus) b += (size_t)n * ld * 4 + (size_t)ld * 4 + (size_t)((ld + 15) & ~15) + (size_t)((n + 15) & ~15) + (size_t)2 * (threads / 32) * 8 + 16;   // replicas of all g_i, grad_i, second selection, branches, distortion partials
     else if (pk_use_table(n, ld, k)) b += (size_t)n * ld * 4;
     if (src == PK_SRC_SMEM) b += (size_t)rows_cta * ld * 4;
     return b;
@@ -610,9 +554,8 @@ PersistPlan plan_persistent(ef21_ctx* c) {
     PersistPlan P; P.ok = false;
     const int ld = (int)c->L.ld;
     if (!c->shards_loaded || ld > 512 || c->k > PK_MAX_K || (i64)c->n * c->k > PK_MAX_MSGS) return P;
-    g_pk_plus = c->variant == EF21_VARIANT_EF21_PLUS;
-    g_pk_ef = c->variant == EF21_VARIANT_EF;
-    if (g_pk_plus && (size_t)c->n * ld * 4 > (size_t)PK_TABLE_MAX_BYTES) return P;      // every block keeps all g_i
+    const bool plus = c->variant == EF21_VARIANT_EF21_PLUS;
+    if (plus && (size_t)c->n * ld * 4 > (size_t)PK_TABLE_MAX_BYTES) return P;      // every block keeps all g_i
     int dev = 0, sms = 0, max_smem = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return P;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -639,7 +582,7 @@ PersistPlan plan_persistent(ef21_ctx* c) {
         }
         if (!rb) {
             rb = max_rb512; threads = 512;
-            src = pk_smem_bytes(c->n, c->k, ld, C, nmsg, PK_SRC_SMEM, rows_cta, threads) <= (size_t)max_smem - 1024 ? PK_SRC_SMEM : PK_SRC_GMEM;
+            src = pk_smem_bytes(plus, c->n, c->k, ld, C, nmsg, PK_SRC_SMEM, rows_cta, threads) <= (size_t)max_smem - 1024 ? PK_SRC_SMEM : PK_SRC_GMEM;
         }
         if (c->pk_threads > 0) {
             threads = c->pk_threads;
@@ -679,9 +622,11 @@ PersistPlan plan_persistent(ef21_ctx* c) {
         const i64 rows_cta = shape_for(C, rb, src, threads, extra);
         if (c->pk_cluster == 0 && C > 1 && rows_cta < 8) continue;       // do not split below one batch
         if (src == PK_SRC_REG && ceil_div(rows_cta, rb + extra) > threads / 32) continue;
-        const size_t smem = pk_smem_bytes(c->n, c->k, ld, C, nmsg, src, rows_cta, threads);
+        const size_t smem = pk_smem_bytes(plus, c->n, c->k, ld, C, nmsg, src, rows_cta, threads);
         if (smem > (size_t)max_smem - 1024) continue;
-        PersistKernel kern = pk_lookup(chunk_slots, rb, src, threads, extra);
+        PersistKernel kern = c->variant == EF21_VARIANT_EF ? pk_lookup_ef(chunk_slots, rb, src, threads, extra)
+                             : (plus ? pk_lookup_plus(chunk_slots, rb, src, threads, extra)
+                                     : pk_lookup_ef21(chunk_slots, rb, src, threads, extra));
         if (!kern) continue;
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
             cudaGetLastError();

@@ -110,36 +110,13 @@ __device__ __forceinline__ void st_async_f4(unsigned remote_dst, float4 v, unsig
 __device__ __forceinline__ float comp_of(const float4& v, int c) {
     return c == 0 ? v.x : (c == 1 ? v.y : (c == 2 ? v.z : v.w));
 }
-#define PK_KERNEL_NAME persistent_kernel
-#define PK_PLUS 0
-#define PK_EF 0
-#include "persistent_body.inc"
-#undef PK_KERNEL_NAME
-#undef PK_PLUS
-#define PK_KERNEL_NAME persistent_plus_kernel
-#define PK_PLUS 1
-#include "persistent_body.inc"
-#undef PK_KERNEL_NAME
-#undef PK_PLUS
-#undef PK_EF
-#define PK_KERNEL_NAME persistent_ef_kernel
-#define PK_PLUS 0
-#define PK_EF 1
-#include "persistent_body.inc"
-#undef PK_KERNEL_NAME
-#undef PK_PLUS
-#undef PK_EF
+typedef void (*PersistKernel)(const PersistParams);
 
-// One-block self-check of the bounded wait: spins on a word that nobody writes and must come back
-// with EF21_ERR_TIMEOUT in the status word instead of hanging.
-__global__ void bounded_wait_selftest_kernel(const unsigned long long* never_written, unsigned* status,
-                                             unsigned spin_limit) {
-    unsigned spins = 0;
-    while (true) {
-        const unsigned long long w = ld_relaxed_u64(never_written);
-        if ((unsigned)(w >> 48) == 0xffffu) break;
-        if (++spins > spin_limit) { record_error(status, 5u); break; }
-    }
-}
+// One lookup per method (each in a translation unit of its own, so that they compile side by side):
+// the kernel instantiated for (chunk slots per lane, rows per warp batch, row source, threads per block,
+// extra rows per batch), or nullptr if that shape is not instantiated.
+PersistKernel pk_lookup_ef21(int chunks, int rb, int src, int threads, int extra);     // Algorithm 2
+PersistKernel pk_lookup_plus(int chunks, int rb, int src, int threads, int extra);     // Algorithm 3
+PersistKernel pk_lookup_ef(int chunks, int rb, int src, int threads, int extra);       // Algorithm 4
 
 }  // namespace ef21

@@ -1,0 +1,6 @@
+// Persistent cluster kernel for the original error feedback method (Algorithm 4): instantiations and their lookup.
+#define PK_KERNEL_NAME persistent_ef_kernel
+#define PK_LOOKUP_NAME pk_lookup_ef
+#define PK_PLUS 0
+#define PK_EF 1
+#include "persistent_method.inc"

@@ -1,0 +1,6 @@
+// Persistent cluster kernel for EF21 (Algorithm 2): instantiations and their lookup.
+#define PK_KERNEL_NAME persistent_kernel
+#define PK_LOOKUP_NAME pk_lookup_ef21
+#define PK_PLUS 0
+#define PK_EF 0
+#include "persistent_method.inc"
