@@ -22,6 +22,12 @@
 //      coordinate thread adds the matching values in ascending worker order (few messages), or warp 0
 //      folds the messages worker by worker into running sums (many messages): g += (1/n) sum c_i
 //
+// The kernel itself is persistent_body.inc; it is compiled three times (persistent_ef21.cu,
+// persistent_plus.cu, persistent_ef.cu): Algorithm 2 as described above, EF21+ (Algorithm 3: a second
+// selection on grad_i, the two distortions, per-block replicas of all g_i and a dense mean) and the
+// original EF (Algorithm 4: the leader compresses e_i + gamma grad_i, the messages move x directly).
+// This header holds what the three share.
+//
 // All summation orders are fixed by the launch shape, so two runs give identical bits.  A wait
 // that exceeds its spin limit records EF21_ERR_TIMEOUT in the status word; from then on every
 // block skips work but keeps arriving at the cluster barriers, so the kernel always terminates.
@@ -110,6 +116,7 @@ __device__ __forceinline__ void st_async_f4(unsigned remote_dst, float4 v, unsig
 __device__ __forceinline__ float comp_of(const float4& v, int c) {
     return c == 0 ? v.x : (c == 1 ? v.y : (c == 2 ? v.z : v.w));
 }
+
 typedef void (*PersistKernel)(const PersistParams);
 
 // One lookup per method (each in a translation unit of its own, so that they compile side by side):
