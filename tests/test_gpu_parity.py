@@ -170,6 +170,30 @@ def test_launch_path_many_steps_in_one_call_equal_single_steps(variant, side_str
             np.testing.assert_array_equal(a_, b_)
 
 
+def test_launch_path_wide_rows_many_steps(B, oracle32):
+    # d = 3,000: two-sweep gradient kernel, one-launch Top-k, two aggregation tiles (offsets recomputed every
+    # iteration, also inside the replayed graph); a multi-step call equals single steps and tracks the oracle
+    rng = np.random.default_rng(77)
+    n, d, k, N = 3, 3000, 30, 600
+    off = np.array([0, 150, 420, 600], dtype=np.int64)
+    A = (rng.standard_normal((N, d)) / np.sqrt(d)).astype(np.float32)
+    y = np.where(rng.random(N) < 0.5, -1.0, 1.0).astype(np.float32)
+    outs = []
+    for chunks in ((8,), (1,) * 8):
+        h = B.EF21(n, d, k, 0.5, 0.1, total_rows=N)
+        h.load_shards(dev(A), dev(y), off)
+        h.init(B.INIT_COMPRESSED)
+        for s_ in chunks:
+            h.step(s_)
+        assert h.last_path == B.PATH_LAUNCHES and h.poll() == 0
+        outs.append(h.get_state_host())
+    for a_, b_ in zip(outs[0], outs[1]):
+        np.testing.assert_array_equal(a_, b_)
+    st = oracle_mod.State(oracle32, n, d, k, 0.5, 0.1, A, y, off)
+    st.init(0); st.step(8)
+    assert rel_l2(outs[0][0], st.x) <= 1e-4
+
+
 def test_eval_matches_oracle(B, oracle32):
     w = inputs.config(0)
     h = make_gpu(w); h.init(B.INIT_COMPRESSED); h.step(5)
