@@ -2,7 +2,7 @@
 """Benchmark of the EF21 hot path (libef21) on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload all|headline|stress|hbm] [--path auto|launches|persistent] [--stress-n N] [--no-cpu] [--no-e2e]
+                    [--workload all|headline|stress|hbm|floor] [--path auto|launches|persistent] [--stress-n N] [--no-cpu] [--no-e2e]
 
 A "step" is one EF21 iteration (Algorithm 2's loop body over all n workers).  The headline
 workload is the mushrooms-shaped logistic problem (n = 20, d = 112, N = 8,124, Top-1, gamma = 1/L);
@@ -32,10 +32,16 @@ METRIC = "EF21 iterations/sec (all n workers, 1 B200) and achieved HBM GB/s vs p
 UNIT = "iterations/s"
 HEADLINE = 1
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes (read + write) of one persistent_kernel launch of 2,000 iterations on the headline workload,
-# from the ncu capture summarised in profiles/persistent_kernel__headline_n20_d112.md.  Reported only for
-# that launch size; None otherwise.
-HEADLINE_TRAFFIC = {"steps": 2000, "bytes": 3749632}
+# Measured DRAM traffic (ncu: dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel, per launch
+# where one launch runs all iterations and per iteration otherwise.  On the on-chip workloads a launch reads the
+# shards and the state from DRAM once, whatever the number of iterations (every later iteration finds its rows in
+# registers, shared memory or L2), so the per-launch figure holds for any step count.  None: not captured for the
+# kernel as it stands.
+NCU_TRAFFIC = {
+    "headline": {"per": "launch", "bytes": None},
+    "hbm_persistent": {"per": "iteration", "bytes": None},
+    "stress_collect": {"per": "iteration", "bytes": None},
+}
 
 
 def logistic_bytes_per_iteration(n, d, k, N):
@@ -148,6 +154,47 @@ def time_oracle(w, steps, warmup):
     return steps / dt, dt, st
 
 
+def host_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def time_oracle_parallel(w, steps, warmup):
+    """The same oracle with the node loop of Algorithm 2 ("for all nodes in parallel") spread over
+    min(n, cores) host threads: every worker's local gradient is one call of the oracle's own routine (the
+    C call runs without the interpreter lock), the message round and the x update stay the oracle's
+    single-threaded code.  Returns (iterations/s, seconds, threads)."""
+    import oracle
+    from concurrent.futures import ThreadPoolExecutor
+    o = oracle.Oracle("f32")
+    st = oracle.State(o, w.n, w.d, w.k, w.gamma, w.lam, w.A, w.y, w.row_offsets, w.x0)
+    st.init(0)
+    threads = max(1, min(w.n, host_cores()))
+    shards = [(w.A[w.row_offsets[i]:w.row_offsets[i + 1]], w.y[w.row_offsets[i]:w.row_offsets[i + 1]]) for i in range(w.n)]
+    grads = np.empty((w.n, w.d), dtype=np.float32)
+
+    def one(i):
+        grads[i] = o.local_grad(shards[i][0], shards[i][1], st.x, w.lam)
+
+    with ThreadPoolExecutor(max_workers=threads) as pool:
+        def iterate(count):
+            for _ in range(count):
+                st.x_update()
+                list(pool.map(one, range(w.n)))
+                st.round(grads)
+        iterate(warmup)
+        t0 = time.perf_counter()
+        iterate(steps)
+        dt = time.perf_counter() - t0
+    return steps / dt, dt, threads
+
+
+def workload_string(w) -> str:
+    return f"configs[{HEADLINE}] {w.name}: n={w.n} d={w.d} N={w.N} Top-{w.k} gamma=1/L lambda={w.lam}"
+
+
 def run_reference(args):
     rank, _, world = dist_env()
     if rank != 0:
@@ -161,7 +208,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": its, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
         "warmup": warmup, "ms_per_step": dt / steps * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64 gradients, f32 state", "data": "synthetic",
-        "config": {"workload": f"configs[{HEADLINE}] {w.name}: n={w.n} d={w.d} N={w.N} Top-{w.k} gamma=1/L"},
+        "config": {"workload": workload_string(w)},
         "cpu_baseline": {"value": its, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": its, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -212,15 +259,18 @@ def run_ours(args):
         hs = B.EF21(n_w, ws.d, ws.k, ws.gamma, device=device)
         hs.init_grads(None, B.INIT_ZERO)
         hs.step_grads(V, max(1, warmup))
-        hs.init_grads(None, B.INIT_ZERO)
-        hs.set_x(torch.zeros(ws.d, dtype=torch.float32, device=device))
-        flush_l2()
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        l0 = hs.launch_count
-        e0.record(); hs.step_grads(V, steps); e1.record()
-        barrier()
-        ms = slowest(e0.elapsed_time(e1))
+        runs = []
+        for _ in range(3):
+            hs.init_grads(None, B.INIT_ZERO)
+            hs.set_x(torch.zeros(ws.d, dtype=torch.float32, device=device))
+            flush_l2()
+            barrier()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            l0 = hs.launch_count
+            e0.record(); hs.step_grads(V, steps); e1.record()
+            barrier()
+            runs.append(slowest(e0.elapsed_time(e1)))
+        ms = statistics.median(runs)
         b = stress_bytes_per_iteration(n_w, ws.d, ws.k)
         gbs = b * steps / (ms * 1e-3) / 1e9
         return {"workload": f"configs[4] {ws.name}: n={n_w} d={ws.d} Top-{ws.k} supplied gradients (static)",
@@ -236,7 +286,7 @@ def run_ours(args):
                               "steps": r["steps"], "ms_per_step": r["us_per_iteration"] / 1e3, "dtype": "f32",
                               "data": "synthetic", "config": {"workload": r["workload"]},
                               "roofline": {"bound": "hbm", "achieved": r["algorithmic_GBps"], "peak": peak, "unit": "GB/s",
-                                           "frac": r["frac_of_hbm_peak"], "traffic": None, "peak_kind": f"of {peak_kind}",
+                                           "frac": r["frac_of_hbm_peak"], "traffic": NCU_TRAFFIC["stress_collect"]["bytes"], "peak_kind": f"of {peak_kind}",
                                            "kernel": "st_collect_kernel (dominant) + sample/finish/aggregate"},
                               "gpu_launches": r["launches"], "fallbacks": r["fallbacks"]}), flush=True)
         if world > 1:
@@ -283,6 +333,27 @@ def run_ours(args):
         return {"ms": ms, "launches": launches, "status": status, "f_end": f_end, "path": h.last_path,
                 "shape": h.get_persistent_shape(), "clocks": sampler.summary() if sampler else None, "handle": h}
 
+    def time_floor(w, k, steps, repeats=5):
+        """us per iteration of the persistent path's exchange skeleton for this shape (no arithmetic of the method)."""
+        h = B.EF21(w.n, w.d, k, w.gamma, w.lam, total_rows=w.N, device=device)
+        h.load_shards(dev(w.A), dev(w.y), w.row_offsets)
+        h.init(B.INIT_COMPRESSED)
+        try:
+            h.selftest_exchange_floor(20)
+        except B.Ef21Error:
+            return None
+        times = []
+        for _ in range(repeats):
+            flush_l2()
+            barrier()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); h.selftest_exchange_floor(steps); e1.record()
+            barrier()
+            times.append(slowest(e0.elapsed_time(e1)))
+        if h.poll() != 0:
+            return None
+        return statistics.median(times) / steps * 1e3
+
     def time_hbm_scale(steps, warmup):
         wb = inputs.hbm_scale_logistic()
         rr = time_logistic(wb, wb.k, steps, warmup)
@@ -294,6 +365,19 @@ def run_ours(args):
                 "algorithmic_bytes_per_iteration": b, "algorithmic_GBps": gbs, "frac_of_hbm_peak": gbs / peak,
                 "launches": rr["launches"], "persistent_shape": rr["shape"], "f_end": rr["f_end"], "device_status": rr["status"]}
 
+    if args.workload == "floor":
+        steps = args.steps if args.steps is not None else 2000
+        rows = []
+        for cfg, k in ((1, 1), (2, 1), (2, 4), (2, 16), (3, 1)):
+            wk = inputs.config(cfg, k=k)
+            rows.append({"workload": f"configs[{cfg}] {wk.name} Top-{k}", "floor_us_per_iteration": time_floor(wk, k, steps)})
+        if rank == 0:
+            print(json.dumps({"metric": "exchange floor of the persistent path (no arithmetic of the method)", "unit": "us per iteration",
+                              "n_gpus": world, "steps": steps, "data": "synthetic", "workloads": rows}), flush=True)
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
     if args.workload == "hbm":
         r = time_hbm_scale(args.steps if args.steps is not None else 50, max(3, args.warmup if args.warmup is not None else 3))
         if rank == 0:
@@ -301,7 +385,8 @@ def run_ours(args):
                               "steps": r["steps"], "ms_per_step": r["us_per_iteration"] / 1e3, "dtype": "f32",
                               "data": "synthetic", "config": {"workload": r["workload"]},
                               "roofline": {"bound": "hbm", "achieved": r["algorithmic_GBps"], "peak": peak, "unit": "GB/s",
-                                           "frac": r["frac_of_hbm_peak"], "traffic": None, "peak_kind": f"of {peak_kind}",
+                                           "frac": r["frac_of_hbm_peak"], "traffic": NCU_TRAFFIC["hbm_persistent"]["bytes"] if args.path != "launches" else None,
+                                           "peak_kind": f"of {peak_kind}",
                                            "kernel": "persistent_kernel, rows streamed from global memory" if args.path != "launches"
                                                      else "grad_stream_kernel (dominant) + per-stage kernels"},
                               "gpu_launches": r["launches"], "persistent_shape": r["persistent_shape"]}), flush=True)
@@ -319,7 +404,9 @@ def run_ours(args):
     achieved = bytes_iter * steps / (r["ms"] * 1e-3) / 1e9
     path_name = {1: "launch-per-stage kernels", 2: "persistent_kernel (one launch for all iterations)"}.get(r["path"], "?")
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": HEADLINE_TRAFFIC["bytes"] if (steps == HEADLINE_TRAFFIC["steps"] and r["path"] == 2) else None,
+                "traffic": NCU_TRAFFIC["headline"]["bytes"] if r["path"] == 2 else None,
+                "traffic_note": "DRAM bytes of one launch (ncu); the same for any number of iterations per launch: the shards "
+                                "and the state are read once, every later iteration finds its rows on chip",
                 "peak_kind": f"of {peak_kind}", "kernel": path_name,
                 "algorithmic_bytes_per_iteration": bytes_iter, "algorithmic_bytes_per_launch": bytes_iter * steps,
                 "note": "latency-bound by design: the 3.6 MB of shards stay on chip, each iteration waits on one "
@@ -350,21 +437,26 @@ def run_ours(args):
         "metric": METRIC, "value": its, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
         "ms_per_step": r["ms"] / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"configs[{HEADLINE}] {w.name}: n={w.n} d={w.d} N={w.N} Top-{w.k} gamma=1/L lambda={w.lam}",
+        "config": {"workload": workload_string(w),
                    "l2": "L2 flushed (256 MB written) before each timed run; inside a run the iterations re-read the same "
                          "shards, which is the method's own access pattern",
                    "replicas": "replicas only: each rank runs the whole n-worker problem" if world > 1 else None,
                    "timed_runs": 5, "value_from": "median run"},
         "roofline": roofline, "e2e": e2e, "gpu_launches": r["launches"], "clocks": r["clocks"],
         "device_status": r["status"], "f_end": r["f_end"], "persistent_shape": r["shape"],
+        "floor_us_per_iteration": time_floor(w, w.k, max(steps, 200)) if r["path"] == 2 else None,
     }
 
     # ---- CPU baseline (rank 0, N = 1 only) ---------------------------------------------------
     if rank == 0 and world == 1 and not args.no_cpu:
         o_steps = min(steps, 2000)
         o_its, o_dt, st = time_oracle(w, o_steps, 3)
+        p_its, p_dt, p_threads = time_oracle_parallel(w, o_steps, 3)
         line["cpu_baseline"] = {"value": o_its, "unit": UNIT, "cores": 1, "kind": "oracle",
-                                "sample": f"{o_steps} full iterations of the headline workload, {o_dt:.1f} s, single thread"}
+                                "sample": f"{o_steps} full iterations of the headline workload, {o_dt:.1f} s, single thread",
+                                "workers_in_parallel": {"value": p_its, "unit": UNIT, "cores": p_threads, "host_cores": host_cores(),
+                                                        "sample": f"{o_steps} full iterations, {p_dt:.1f} s; the node loop of Algorithm 2 on "
+                                                                  f"{p_threads} threads (one oracle gradient call per worker), the rest single-threaded"}}
     else:
         line["cpu_baseline"] = None
 
@@ -377,7 +469,8 @@ def run_ours(args):
             b = logistic_bytes_per_iteration(wk.n, wk.d, k, wk.N)
             gbs = b * wk.T / (rr["ms"] * 1e-3) / 1e9
             others.append({"workload": f"configs[{cfg}] {wk.name} Top-{k}", "iterations_per_s": wk.T / (rr["ms"] * 1e-3),
-                           "us_per_iteration": rr["ms"] / wk.T * 1e3, "algorithmic_GBps": gbs, "frac_of_hbm_peak": gbs / peak,
+                           "us_per_iteration": rr["ms"] / wk.T * 1e3, "algorithmic_bytes_per_iteration": b, "algorithmic_GBps": gbs,
+                           "frac_of_hbm_peak": gbs / peak, "floor_us_per_iteration": time_floor(wk, k, wk.T) if rr["path"] == 2 else None,
                            "launches": rr["launches"], "persistent_shape": rr["shape"], "f_end": rr["f_end"]})
         others.append(time_stress(None, 50, 3))
         others.append(time_hbm_scale(50, 3))
@@ -391,6 +484,9 @@ def run_ours(args):
         others.append({"workload": f"EF (Algorithm 4) on configs[{HEADLINE}] {wp.name} Top-{wp.k}", "iterations_per_s": 500 / (re_["ms"] * 1e-3),
                        "us_per_iteration": re_["ms"] / 500 * 1e3, "launches": re_["launches"], "f_end": re_["f_end"]})
         line["workloads"] = others
+        line["workloads_note"] = ("frac_of_hbm_peak = algorithmic bytes per iteration / time / measured copy peak (read + write); on the "
+                                  "on-chip workloads it is not a DRAM figure (DRAM traffic per launch is the shards once), and a read-only "
+                                  "stream can exceed a copy peak slightly")
 
     if world > 1:
         dist.destroy_process_group()
@@ -404,10 +500,11 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="all", choices=["all", "headline", "stress", "hbm"],
+    ap.add_argument("--workload", default="all", choices=["all", "headline", "stress", "hbm", "floor"],
                     help="all: headline line with the other workloads attached; headline: only the headline; "
                          "stress: only the supplied-gradient workload; hbm: only the logistic workload whose shards "
-                         "exceed L2 (each its own line; for profiling)")
+                         "exceed L2 (each its own line; for profiling); floor: the exchange skeleton of the persistent "
+                         "path on the logistic workloads")
     ap.add_argument("--path", default="auto", choices=["auto", "launches", "persistent"],
                     help="execution path of the logistic workloads (default: the library's own choice)")
     ap.add_argument("--stress-n", type=int, default=None, help="workers of the stress workload (default 64)")

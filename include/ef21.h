@@ -198,26 +198,42 @@ ef21_status ef21_get_state_host(ef21_ctx* ctx, float* x_host, float* g_host, flo
 ef21_status ef21_set_state(ef21_ctx* ctx, const float* x_dev, const float* g_dev, const float* gi_dev);
 
 /* Diagnostics at the current state (synchronises): f(x) of Eq. 19 / Eq. 1, ||grad f(x)||^2,
- * and G^t = (1/n) sum_i ||g_i - grad f_i(x)||^2 of Section 3.3.  Any pointer may be NULL. */
+ * and G^t = (1/n) sum_i ||g_i - grad f_i(x)||^2 of Section 3.3.  Any pointer may be NULL.  If one of
+ * the three is NaN or Inf the values are still written and EF21_ERR_NONFINITE is returned. */
 ef21_status ef21_eval(ef21_ctx* ctx, double* f, double* grad_norm2, double* G);
 
 /* Synchronises the stream and returns the device status word: EF21_OK, or the first
- * error a kernel recorded (EF21_ERR_TIMEOUT, EF21_ERR_NONFINITE), or EF21_ERR_CUDA. */
+ * error a kernel recorded, or EF21_ERR_CUDA.
+ *   EF21_ERR_NONFINITE: a compressor of this handle (init, step, step_grads, step_minibatch, any
+ *     method) selected a NaN or Inf.  The compressor of Section 2.1 is defined on real vectors; a
+ *     non-finite entry has the largest key (bit-pattern order), so it is always selected and one
+ *     anywhere in a compressed vector -- a supplied gradient, or a gradient at a non-finite x -- is
+ *     noticed in the step that meets it.  The state is unspecified from that step on: restore it with
+ *     ef21_set_state and call ef21_clear_status.  The standalone ef21_topk has no status word and does
+ *     not check.
+ *   EF21_ERR_TIMEOUT: a bounded wait of the persistent kernel expired (its clusters were not all
+ *     running at once, e.g. another kernel of the process held SMs).  The blocks leave the iteration
+ *     loop at different iterations, so the state (x, g, g_i, last messages) is unspecified afterwards:
+ *     restore it with ef21_set_state, call ef21_clear_status, and use EF21_PATH_LAUNCHES if the
+ *     device stays shared.
+ *   EF21_ERR_INVALID_ARG: ef21_step_minibatch met a row number outside its shard. */
 ef21_status ef21_poll(ef21_ctx* ctx);
 
 /* Selects the local objective (EF21_OBJECTIVE_*) used by ef21_init, ef21_step, ef21_local_grads and
  * ef21_eval; default logistic.  Both execution paths support both objectives. */
 ef21_status ef21_set_objective(ef21_ctx* ctx, int32_t objective);
 
-/* EF21+ (Section 3.4, Algorithm 3).  With EF21_VARIANT_EF21_PLUS every step computes, per worker,
+/* Selects the method (EF21_VARIANT_*) that ef21_step / ef21_step_grads run; default Algorithm 2.
+ *
+ * EF21+ (Section 3.4, Algorithm 3).  With EF21_VARIANT_EF21_PLUS every step computes, per worker,
  * b_i = C(grad f_i(x)) and m_i = g_i + C(grad f_i(x) - g_i), the distortions B_i = ||b_i - grad f_i(x)||^2
  * and M_i = ||m_i - grad f_i(x)||^2 (fp64 sums of the fp32 vectors), sets g_i = m_i if M_i <= B_i and
  * g_i = b_i otherwise, and recomputes g = (1/n) sum_i g_i (ascending i, then one multiply).  Both
  * execution paths run it; the persistent kernel needs n * d * 4 <= 64 KB (every block keeps a copy
  * of all g_i), otherwise the launch path is taken.  The "last message" of ef21_get_state is the
- * compressed vector that was used.  Initialisation is that of Algorithm 2. */
-ef21_status ef21_set_variant(ef21_ctx* ctx, int32_t variant);
-/* The original error feedback method, EF (Section 4.1, Algorithm 4), with EF21_VARIANT_EF.  The
+ * compressed vector that was used.  Initialisation is that of Algorithm 2.
+ *
+ * The original error feedback method, EF (Section 4.1, Algorithm 4), with EF21_VARIANT_EF.  The
  * per-worker state is the error e_i, kept where Algorithm 2 keeps g_i (the gi argument of
  * ef21_get_state / ef21_set_state); g is not used.  Algorithm 4 starts from e_i^0 = 0: call
  * ef21_init(ctx, EF21_INIT_ZERO).  One step from (x^t, e_i^t) computes
@@ -230,6 +246,7 @@ ef21_status ef21_set_variant(ef21_ctx* ctx, int32_t variant);
  * operations; the sum over workers runs in ascending worker order.  ef21_step_grads uses the
  * supplied vectors in place of grad f_i.  Both execution paths run ef21_step; ef21_step_minibatch
  * is not available. */
+ef21_status ef21_set_variant(ef21_ctx* ctx, int32_t variant);
 /* choice_host[n]: 0 where the last EF21+ step kept the Markov compressor, 1 where it took C(grad);
  * synchronises. */
 ef21_status ef21_get_plus_choice(ef21_ctx* ctx, int32_t* choice_host);
@@ -250,6 +267,15 @@ ef21_status ef21_clear_status(ef21_ctx* ctx);
  * at most spin_limit (1 .. 2^24) times on a word that nothing writes, then records
  * EF21_ERR_TIMEOUT, which the next ef21_poll returns.  The device and the context stay usable. */
 ef21_status ef21_selftest_bounded_wait(ef21_ctx* ctx, uint32_t spin_limit);
+
+/* Measuring aid: `steps` iterations of the persistent path's exchange skeleton for this handle's shape -- the
+ * same clusters, barriers, hand-off of the block partials to the cluster leader, publication and polling
+ * of the n*k message words, every wait bounded as in ef21_step -- with all arithmetic of the method left
+ * out (no row sweep, no selection, no aggregation).  The state is not touched.  Timing it gives the cost
+ * of the two dependencies Algorithm 2 has per iteration (broadcast of x^{t+1}, collection of the c_i^t) on
+ * this device, a floor under the iteration time of ef21_step.  EF21_ERR_UNSUPPORTED if the shape has no
+ * persistent path. */
+ef21_status ef21_selftest_exchange_floor(ef21_ctx* ctx, int32_t steps);
 
 /* Tuning of the persistent path (Algorithm 2 as one kernel; worker i = one thread-block
  * cluster): blocks per cluster (1..8, 0 = automatic), rows per warp batch (4, 8, 16, 32, 0 =

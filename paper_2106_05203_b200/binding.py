@@ -57,6 +57,7 @@ SIGNATURES = {
     "ef21_fallback_count": (ctypes.c_int, [_vp, ctypes.POINTER(_i64)]),
     "ef21_clear_status": (ctypes.c_int, [_vp]),
     "ef21_selftest_bounded_wait": (ctypes.c_int, [_vp, ctypes.c_uint32]),
+    "ef21_selftest_exchange_floor": (ctypes.c_int, [_vp, ctypes.c_int32]),
     "ef21_set_persistent_shape": (ctypes.c_int, [_vp, _i32, _i32, _i32]),
     "ef21_get_persistent_shape": (ctypes.c_int, [_vp, ctypes.POINTER(_i32), ctypes.POINTER(_i32), ctypes.POINTER(_i32)]),
     "ef21_set_persistent_threads": (ctypes.c_int, [_vp, _i32]),
@@ -268,6 +269,9 @@ class EF21:
 
     def selftest_bounded_wait(self, spin_limit: int) -> None:
         _check(_lib.ef21_selftest_bounded_wait(self._h, spin_limit), "ef21_selftest_bounded_wait")
+
+    def selftest_exchange_floor(self, steps: int) -> None:
+        _check(_lib.ef21_selftest_exchange_floor(self._h, steps), "ef21_selftest_exchange_floor")
 
     def set_persistent_shape(self, cluster_blocks: int = 0, rows_per_batch: int = 0, row_source: int = -1) -> None:
         _check(_lib.ef21_set_persistent_shape(self._h, cluster_blocks, rows_per_batch, row_source),

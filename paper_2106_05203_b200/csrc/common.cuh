@@ -16,6 +16,13 @@ __device__ __forceinline__ void record_error(unsigned* status, unsigned code) {
 // order of magnitudes; +0 and -0 share key 0.
 __device__ __forceinline__ unsigned mag_key(float v) { return __float_as_uint(v) & 0x7fffffffu; }
 
+// Non-finite inputs of the compressor: a NaN or Inf has a key above every finite value's, so it is always
+// among the k selected entries -- checking the selected values is enough to notice one anywhere in the vector.
+// Records EF21_ERR_NONFINITE in the status word (status may be null: standalone calls have none).
+__device__ __forceinline__ void flag_nonfinite(unsigned* status, float selected) {
+    if (status != nullptr && mag_key(selected) > 0x7f7fffffu) record_error(status, 6u /* EF21_ERR_NONFINITE */);
+}
+
 // v = a - b as one rounded fp32 subtraction (b == nullptr: v = a).
 __device__ __forceinline__ float diff_at(const float* __restrict__ a, const float* __restrict__ b, i64 j) {
     float av = a[j];

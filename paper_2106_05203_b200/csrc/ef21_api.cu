@@ -41,16 +41,25 @@ struct TopkLayout {
 
 bool fast_topk_eligible(i64 d, i64 k) { return d >= ST_MIN_D && k <= ST_MAX_K; }
 
-TopkLayout topk_layout(i64 batch, i64 d, i64 k) {
-    TopkLayout L;
+// The three sections every Top-k call needs (selection state, histogram, per-chunk counts); the
+// one-pass sections are absent.
+TopkLayout topk_layout_general(i64 batch, i64 d) {
+    TopkLayout L{};
     L.nchunks = (int)ceil_div(d, TK_CHUNK);
     size_t o = 0;
     L.state = o; o += align_up((size_t)batch * sizeof(TkState));
     L.hist = o; o += align_up((size_t)batch * TK_BINS * sizeof(unsigned));
     L.chunks = o; o += align_up((size_t)batch * (size_t)L.nchunks * sizeof(uint2));
-    L.fast = fast_topk_eligible(d, k);
+    L.fast = false;
     L.nreg = (int)ceil_div(d, ST_SUB);
-    L.thr = L.flags = L.done = L.slow_count = L.region_cnt = L.cand = 0;
+    L.total = o;
+    return L;
+}
+
+TopkLayout topk_layout(i64 batch, i64 d, i64 k) {
+    TopkLayout L = topk_layout_general(batch, d);
+    size_t o = L.total;
+    L.fast = fast_topk_eligible(d, k);
     if (L.fast) {
         L.thr = o; o += align_up((size_t)batch * 4);
         L.flags = o; o += align_up((size_t)batch * 4);
@@ -242,13 +251,21 @@ ef21_status enqueue_topk_fast_sample(cudaStream_t st, const float* a, i64 pitch_
 // is given, g_i += c_i is applied by the same kernel that writes the messages.
 ef21_status enqueue_topk_fast(cudaStream_t st, const float* a, i64 pitch_a, const float* b, i64 pitch_b,
                               int batch, i64 d, int k, int* idx_out, float* val_out, float* gi_rows, i64 ld,
-                              const TopkBuffers& B, i64* launches, bool sampled = false, int* tile_off = nullptr,
-                              int ntiles = 0) {
-    static bool smem_set = false;
+                              const TopkBuffers& B, i64* launches, unsigned* status, bool sampled = false,
+                              int* tile_off = nullptr, int ntiles = 0) {
     const size_t finish_smem = (size_t)ST_CAND_CAP * 12 + 2048 * 4;
-    if (!smem_set) {
-        CU(cudaFuncSetAttribute(st_finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)finish_smem));
-        smem_set = true;
+    {
+        // the shared-memory opt-in is a per-device attribute of the kernel: set once per device ordinal
+        constexpr int MAX_DEVICES = 64;
+        static std::mutex mu;
+        static bool smem_set[MAX_DEVICES] = {};
+        int dev = -1;
+        CU(cudaGetDevice(&dev));
+        std::lock_guard<std::mutex> lock(mu);
+        if (dev < 0 || dev >= MAX_DEVICES || !smem_set[dev]) {
+            CU(cudaFuncSetAttribute(st_finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)finish_smem));
+            if (dev >= 0 && dev < MAX_DEVICES) smem_set[dev] = true;
+        }
     }
     if (!sampled) EF(enqueue_topk_fast_sample(st, a, pitch_a, b, pitch_b, batch, d, k, B, launches));
     dim3 grid((unsigned)ceil_div(B.nreg, ST_COLLECT_WARPS), (unsigned)batch);
@@ -257,7 +274,7 @@ ef21_status enqueue_topk_fast(cudaStream_t st, const float* a, i64 pitch_a, cons
     collect<<<grid, ST_COLLECT_WARPS * 32, 0, st>>>(a, pitch_a, b, pitch_b, d, B.nreg, B.thr, B.cand, B.region_cnt, B.flags);
     st_finish_kernel<<<batch, ST_THREADS, finish_smem, st>>>(a, pitch_a, b, pitch_b, d, B.nreg, k, B.cand, B.region_cnt,
                                                              B.flags, idx_out, val_out, gi_rows, ld, B.slow_count, tile_off,
-                                                             ntiles, AGG_TILE);
+                                                             ntiles, AGG_TILE, status);
     if (launches) *launches += 2;
     CU(cudaGetLastError());
     return EF21_OK;
@@ -266,14 +283,14 @@ ef21_status enqueue_topk_fast(cudaStream_t st, const float* a, i64 pitch_a, cons
 // Exact Top-k of v = a - b for `batch` vectors (b may be null); general multi-block path.
 ef21_status enqueue_topk_general(cudaStream_t st, const float* a, i64 pitch_a, const float* b, i64 pitch_b,
                                  int batch, i64 d, int k, int* idx_out, float* val_out,
-                                 const TopkBuffers& B, i64* launches, float* apply_to = nullptr, i64 pitch_apply = 0,
-                                 bool* applied = nullptr) {
+                                 const TopkBuffers& B, i64* launches, unsigned* status, float* apply_to = nullptr,
+                                 i64 pitch_apply = 0, bool* applied = nullptr) {
     if (applied) *applied = false;
     if (d <= TKS_MAX_D) {
         // short vectors: the whole selection in one launch, one block per vector (no scratch); the same
         // launch adds the messages to apply_to if the caller asks for it
         tk_small_kernel<<<batch, TKS_BLOCK, (size_t)d * 4, st>>>(a, pitch_a, b, pitch_b, (int)d, k, idx_out, val_out,
-                                                                 apply_to, pitch_apply);
+                                                                 apply_to, pitch_apply, status);
         if (applied) *applied = apply_to != nullptr;
         if (launches) *launches += 1;
         CU(cudaGetLastError());
@@ -288,7 +305,7 @@ ef21_status enqueue_topk_general(cudaStream_t st, const float* a, i64 pitch_a, c
     tk_count_kernel<<<grid, TK_BLOCK, 0, st>>>(a, pitch_a, b, pitch_b, d, B.state, B.chunks, B.nchunks);
     tk_scan_kernel<<<batch, 1024, 0, st>>>(B.chunks, B.nchunks);
     tk_write_kernel<<<grid, TK_BLOCK, 0, st>>>(a, pitch_a, b, pitch_b, d, B.state, B.chunks, B.nchunks, k,
-                                               idx_out, val_out);
+                                               idx_out, val_out, status);
     if (launches) *launches += 10;
     CU(cudaGetLastError());
     return EF21_OK;
@@ -365,13 +382,13 @@ ef21_status enqueue_round_select(ef21_ctx* c, const float* a, i64 pitch_a, bool 
     if (B.fast && !c->force_general_topk) {
         // the finish kernel also leaves the per-tile offsets of the messages for the aggregation
         EF(enqueue_topk_fast(c->stream, a, pitch_a, c->gi(), c->L.ld, c->n, c->d, c->k, c->msg_idx(), c->msg_val(),
-                             c->gi(), c->L.ld, B, &c->launches, sampled, c->at<int>(c->L.agg_off), c->L.agg_tiles));
+                             c->gi(), c->L.ld, B, &c->launches, c->status(), sampled, c->at<int>(c->L.agg_off), c->L.agg_tiles));
         c->agg_off_ready = true;
     } else {
         c->agg_off_ready = false;
         bool applied = false;
         EF(enqueue_topk_general(c->stream, a, pitch_a, c->gi(), c->L.ld, c->n, c->d, c->k, c->msg_idx(),
-                                c->msg_val(), B, &c->launches, c->gi(), c->L.ld, &applied));
+                                c->msg_val(), B, &c->launches, c->status(), c->gi(), c->L.ld, &applied));
         if (!applied) {
             const i64 total = (i64)c->n * c->k;
             apply_messages_kernel<<<(unsigned)ceil_div(total, 256), 256, 0, c->stream>>>(c->msg_idx(), c->msg_val(), total,
@@ -423,12 +440,12 @@ ef21_status enqueue_plus_round(ef21_ctx* c, const float* a, i64 pitch_a) {
     float* val_b = c->at<float>(c->L.msg2_val);
     if (B.fast && !c->force_general_topk) {
         EF(enqueue_topk_fast(c->stream, a, pitch_a, c->gi(), c->L.ld, c->n, c->d, c->k, c->msg_idx(), c->msg_val(),
-                             nullptr, 0, B, &c->launches));
-        EF(enqueue_topk_fast(c->stream, a, pitch_a, nullptr, 0, c->n, c->d, c->k, idx_b, val_b, nullptr, 0, B, &c->launches));
+                             nullptr, 0, B, &c->launches, c->status()));
+        EF(enqueue_topk_fast(c->stream, a, pitch_a, nullptr, 0, c->n, c->d, c->k, idx_b, val_b, nullptr, 0, B, &c->launches, c->status()));
     } else {
         EF(enqueue_topk_general(c->stream, a, pitch_a, c->gi(), c->L.ld, c->n, c->d, c->k, c->msg_idx(), c->msg_val(), B,
-                                &c->launches));
-        EF(enqueue_topk_general(c->stream, a, pitch_a, nullptr, 0, c->n, c->d, c->k, idx_b, val_b, B, &c->launches));
+                                &c->launches, c->status()));
+        EF(enqueue_topk_general(c->stream, a, pitch_a, nullptr, 0, c->n, c->d, c->k, idx_b, val_b, B, &c->launches, c->status()));
     }
     plus_choose_kernel<<<c->n, PLUS_BLOCK, 0, c->stream>>>(a, pitch_a, c->gi(), c->L.ld, c->d, c->k, c->msg_idx(), c->msg_val(),
                                                           idx_b, val_b, c->at<float>(c->L.plus_old), c->at<unsigned>(c->L.plus_bitmap),
@@ -450,10 +467,10 @@ ef21_status enqueue_ef_round(ef21_ctx* c, const float* a, i64 pitch_a) {
     c->launches += 1;
     if (B.fast && !c->force_general_topk) {
         EF(enqueue_topk_fast(c->stream, c->gi(), c->L.ld, nullptr, 0, c->n, c->d, c->k, c->msg_idx(), c->msg_val(),
-                             nullptr, 0, B, &c->launches));
+                             nullptr, 0, B, &c->launches, c->status()));
     } else {
         EF(enqueue_topk_general(c->stream, c->gi(), c->L.ld, nullptr, 0, c->n, c->d, c->k, c->msg_idx(), c->msg_val(), B,
-                                &c->launches));
+                                &c->launches, c->status()));
     }
     const i64 total = (i64)c->n * c->k;
     ef_subtract_sent_kernel<<<(unsigned)ceil_div(total, 256), 256, 0, c->stream>>>(c->msg_idx(), c->msg_val(), total, c->k,
@@ -515,6 +532,8 @@ ef21_status finish_load(ef21_ctx* c, const i64* row_offsets_host) {
     c->tile_begin[c->n] = (int)c->tiles.size();
     c->num_tiles = (int)c->tiles.size();
     if ((i64)c->num_tiles > c->L.max_tiles) return EF21_ERR_WORKSPACE;
+    // a captured launch-path iteration has the old tile count baked into its grid
+    if (c->iter_graph) { cudaGraphExecDestroy(c->iter_graph); c->iter_graph = nullptr; }
     CU(cudaMemcpyAsync(c->at<i64>(c->L.row_off), c->row_off.data(), (size_t)(c->n + 1) * 8, cudaMemcpyHostToDevice, c->stream));
     CU(cudaMemcpyAsync(c->at<int>(c->L.tile_begin), c->tile_begin.data(), (size_t)(c->n + 1) * 4, cudaMemcpyHostToDevice, c->stream));
     if (c->num_tiles > 0)
@@ -550,7 +569,7 @@ size_t pk_smem_bytes(bool plus, int n, int k, int ld, int C, int nmsg, int src, 
 
 // Chooses cluster size, block size, rows per batch and the source of the shard rows; checks that all n
 // clusters can be resident at once (the blocks wait on one another through global memory).
-PersistPlan plan_persistent(ef21_ctx* c) {
+PersistPlan plan_persistent(ef21_ctx* c, bool floor_only = false) {
     PersistPlan P; P.ok = false;
     const int ld = (int)c->L.ld;
     if (!c->shards_loaded || ld > 512 || c->k > PK_MAX_K || (i64)c->n * c->k > PK_MAX_MSGS) return P;
@@ -624,7 +643,8 @@ PersistPlan plan_persistent(ef21_ctx* c) {
         if (src == PK_SRC_REG && ceil_div(rows_cta, rb + extra) > threads / 32) continue;
         const size_t smem = pk_smem_bytes(plus, c->n, c->k, ld, C, nmsg, src, rows_cta, threads);
         if (smem > (size_t)max_smem - 1024) continue;
-        PersistKernel kern = c->variant == EF21_VARIANT_EF ? pk_lookup_ef(chunk_slots, rb, src, threads, extra)
+        PersistKernel kern = floor_only ? pk_lookup_floor(chunk_slots, rb, src, threads, extra)
+                             : c->variant == EF21_VARIANT_EF ? pk_lookup_ef(chunk_slots, rb, src, threads, extra)
                              : (plus ? pk_lookup_plus(chunk_slots, rb, src, threads, extra)
                                      : pk_lookup_ef21(chunk_slots, rb, src, threads, extra));
         if (!kern) continue;
@@ -972,8 +992,8 @@ ef21_status ef21_topk(const float* v_dev, int32_t batch, int64_t d, int32_t k, i
     TopkBuffers B = topk_buffers(static_cast<char*>(workspace_dev), L);
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
     if (B.fast)
-        return enqueue_topk_fast(st, v_dev, d, nullptr, 0, batch, d, k, idx_out_dev, val_out_dev, nullptr, 0, B, nullptr);
-    return enqueue_topk_general(st, v_dev, d, nullptr, 0, batch, d, k, idx_out_dev, val_out_dev, B, nullptr);
+        return enqueue_topk_fast(st, v_dev, d, nullptr, 0, batch, d, k, idx_out_dev, val_out_dev, nullptr, 0, B, nullptr, nullptr);
+    return enqueue_topk_general(st, v_dev, d, nullptr, 0, batch, d, k, idx_out_dev, val_out_dev, B, nullptr, nullptr);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1012,14 +1032,7 @@ ef21_status ef21_topk_static(const float* v_dev, int32_t batch, int64_t d, int32
     if (!v_dev || !idx_out_dev || !val_out_dev || batch < 1 || !valid_shape(1, d, k, 0)) return EF21_ERR_INVALID_ARG;
     if (batch > TOPK_STATIC_MAX_BATCH || (i64)batch * ceil_div(d, TK_CHUNK) > TOPK_STATIC_MAX_CHUNKS)
         return EF21_ERR_UNSUPPORTED;                     // beyond the built-in scratch
-    TopkLayout L;
-    L.nchunks = (int)ceil_div(d, TK_CHUNK);
-    size_t o = 0;
-    L.state = o; o += align_up((size_t)batch * sizeof(TkState));
-    L.hist = o; o += align_up((size_t)batch * TK_BINS * sizeof(unsigned));
-    L.chunks = o; o += align_up((size_t)batch * (size_t)L.nchunks * sizeof(uint2));
-    L.fast = false; L.nreg = 0; L.thr = L.flags = L.slow_count = L.region_cnt = L.cand = 0;
-    L.total = o;
+    const TopkLayout L = topk_layout_general(batch, d);      // the same three sections ef21_topk lays out
     if (L.total > TOPK_STATIC_SCRATCH_BYTES) return EF21_ERR_UNSUPPORTED;
     void* scratch = nullptr;
     EF(topk_static_scratch(&scratch));
@@ -1027,7 +1040,7 @@ ef21_status ef21_topk_static(const float* v_dev, int32_t batch, int64_t d, int32
     // tk_reset_kernel clears the selection state and the histograms of the vectors in use; the
     // per-chunk counts are fully rewritten before they are read.
     return enqueue_topk_general(reinterpret_cast<cudaStream_t>(cuda_stream), v_dev, d, nullptr, 0, batch, d, k,
-                                idx_out_dev, val_out_dev, B, nullptr);
+                                idx_out_dev, val_out_dev, B, nullptr, nullptr);
 }
 
 static ef21_status copy_state_out(ef21_ctx* c, float* x, float* g, float* gi, int32_t* li, float* lv, cudaMemcpyKind kind) {
@@ -1076,6 +1089,7 @@ ef21_status ef21_eval(ef21_ctx* c, double* f, double* grad_norm2, double* G) {
     if (f) *f = out[0];
     if (grad_norm2) *grad_norm2 = out[1];
     if (G) *G = out[2];
+    if (!std::isfinite(out[0]) || !std::isfinite(out[1]) || !std::isfinite(out[2])) return EF21_ERR_NONFINITE;
     return EF21_OK;
 }
 
@@ -1167,6 +1181,15 @@ ef21_status ef21_selftest_bounded_wait(ef21_ctx* c, uint32_t spin_limit) {
     c->launches += 1;
     CU(cudaGetLastError());
     return EF21_OK;
+}
+
+ef21_status ef21_selftest_exchange_floor(ef21_ctx* c, int32_t steps) {
+    if (!c || steps < 1) return EF21_ERR_INVALID_ARG;
+    if (!c->shards_loaded || !c->inited) return EF21_ERR_STATE;
+    if (c->variant != EF21_VARIANT_EF21) return EF21_ERR_UNSUPPORTED;
+    PersistPlan P = plan_persistent(c, true);
+    if (!P.ok) return EF21_ERR_UNSUPPORTED;
+    return run_persistent(c, P, steps);
 }
 
 int32_t ef21_last_path(const ef21_ctx* c) { return c ? c->last_path : 0; }

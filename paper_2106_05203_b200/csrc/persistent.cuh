@@ -125,5 +125,6 @@ typedef void (*PersistKernel)(const PersistParams);
 PersistKernel pk_lookup_ef21(int chunks, int rb, int src, int threads, int extra);     // Algorithm 2
 PersistKernel pk_lookup_plus(int chunks, int rb, int src, int threads, int extra);     // Algorithm 3
 PersistKernel pk_lookup_ef(int chunks, int rb, int src, int threads, int extra);       // Algorithm 4
+PersistKernel pk_lookup_floor(int chunks, int rb, int src, int threads, int extra);    // exchange skeleton (measuring aid)
 
 }  // namespace ef21

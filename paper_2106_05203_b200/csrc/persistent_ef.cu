@@ -3,4 +3,5 @@
 #define PK_LOOKUP_NAME pk_lookup_ef
 #define PK_PLUS 0
 #define PK_EF 1
+#define PK_FLOOR 0
 #include "persistent_method.inc"

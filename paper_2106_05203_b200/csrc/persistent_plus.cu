@@ -3,4 +3,5 @@
 #define PK_LOOKUP_NAME pk_lookup_plus
 #define PK_PLUS 1
 #define PK_EF 0
+#define PK_FLOOR 0
 #include "persistent_method.inc"

@@ -116,7 +116,7 @@ __device__ __forceinline__ bool select_match(unsigned key, int level, unsigned p
 // Whole-vector exact Top-k by one block (fallback): three histogram passes, one ordered pass.
 __device__ void st_slow_exact(const float* av, const float* bv, i64 d, int k,
                               int* __restrict__ idx_out, float* __restrict__ val_out, float* gi_row,
-                              unsigned* hist, unsigned* scratch, unsigned* res) {
+                              unsigned* hist, unsigned* scratch, unsigned* res, unsigned* status) {
     SelectState s; s.prefix = 0u; s.need = (unsigned)k; s.lo_ge = 0u; s.T = 0u; s.need_ties = 0u; s.done = 0u;
     for (int level = 0; level < 3 && !s.done; ++level) {
         for (int q = threadIdx.x; q < 2048; q += ST_THREADS) hist[q] = 0u;
@@ -148,6 +148,7 @@ __device__ void st_slow_exact(const float* av, const float* bv, i64 d, int k,
             const unsigned pos = is_ge ? my_ge + min(my_tie, s.need_ties) : my_ge + my_tie;
             if (pos < (unsigned)k) {
                 idx_out[pos] = (int)j; val_out[pos] = val;
+                flag_nonfinite(status, val);
                 if (gi_row) gi_row[j] = __fadd_rn(gi_row[j], val);
             }
         }
@@ -246,7 +247,7 @@ st_finish_kernel(const float* a, i64 pitch_a, const float* b, i64 pitch_b, i64 d
                  const int4* __restrict__ cand, const int* __restrict__ region_cnt,
                  const unsigned* __restrict__ flags, int* __restrict__ idx_out, float* __restrict__ val_out,
                  float* gi_rows, i64 ld, unsigned* __restrict__ slow_count,
-                 int* __restrict__ tile_off, int ntiles, int tile) {
+                 int* __restrict__ tile_off, int ntiles, int tile, unsigned* status) {
     extern __shared__ __align__(16) unsigned char st_smem[];
     __shared__ unsigned scratch[33];
     __shared__ unsigned res[3];
@@ -305,7 +306,7 @@ st_finish_kernel(const float* a, i64 pitch_a, const float* b, i64 pitch_b, i64 d
     }
     if (bad || total < (unsigned)k || total > (unsigned)ST_CAND_CAP) {
         if (threadIdx.x == 0 && slow_count) atomicAdd(slow_count, 1u);
-        st_slow_exact(av, bv, d, k, io, vo, gi_row, hist, scratch, res);
+        st_slow_exact(av, bv, d, k, io, vo, gi_row, hist, scratch, res, status);
         if (tile_off) {
             __syncthreads();                         // the block's own writes to io are visible to it now
             int* off = tile_off + (i64)i * (ntiles + 1);
@@ -374,6 +375,7 @@ st_finish_kernel(const float* a, i64 pitch_a, const float* b, i64 pitch_b, i64 d
     for (int p0 = threadIdx.x; p0 < k; p0 += ST_THREADS) {
         const int2 me = out2[p0];
         io[p0] = me.x; vo[p0] = __int_as_float(me.y);
+        flag_nonfinite(status, __int_as_float(me.y));
         if (off) {
             const int t_prev = p0 > 0 ? out2[p0 - 1].x / tile : -1;
             const int t_me = me.x / tile;

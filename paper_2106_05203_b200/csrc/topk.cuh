@@ -159,7 +159,7 @@ tk_scan_kernel(uint2* __restrict__ chunk_counts, int nchunks) {
 __global__ void __launch_bounds__(TK_BLOCK)
 tk_write_kernel(const float* __restrict__ a, i64 pitch_a, const float* __restrict__ b, i64 pitch_b, i64 d,
                 const TkState* __restrict__ st, const uint2* __restrict__ chunk_prefix, int nchunks,
-                int k, int* __restrict__ idx_out, float* __restrict__ val_out) {
+                int k, int* __restrict__ idx_out, float* __restrict__ val_out, unsigned* status) {
     __shared__ unsigned scratch[33];
     const int v = blockIdx.y;
     const TkState s = st[v];
@@ -186,10 +186,10 @@ tk_write_kernel(const float* __restrict__ a, i64 pitch_a, const float* __restric
         const unsigned my_tie = tie_before + (packed >> 16);
         if (is_ge) {
             const unsigned pos = my_ge + min(my_tie, s.need_ties);
-            if (pos < (unsigned)k) { io[pos] = (int)j; vo[pos] = val; }
+            if (pos < (unsigned)k) { io[pos] = (int)j; vo[pos] = val; flag_nonfinite(status, val); }
         } else if (is_tie && my_tie < s.need_ties) {
             const unsigned pos = my_ge + my_tie;
-            if (pos < (unsigned)k) { io[pos] = (int)j; vo[pos] = val; }
+            if (pos < (unsigned)k) { io[pos] = (int)j; vo[pos] = val; flag_nonfinite(status, val); }
         }
         ge_before += tot & 0xffffu;
         tie_before += tot >> 16;
@@ -211,7 +211,8 @@ constexpr int TKS_BLOCK = 512;
 
 __global__ void __launch_bounds__(TKS_BLOCK)
 tk_small_kernel(const float* __restrict__ a, i64 pitch_a, const float* b, i64 pitch_b,
-                int d, int k, int* __restrict__ idx_out, float* __restrict__ val_out, float* apply_to, i64 pitch_apply) {
+                int d, int k, int* __restrict__ idx_out, float* __restrict__ val_out, float* apply_to, i64 pitch_apply,
+                unsigned* status) {
     extern __shared__ __align__(16) unsigned char tks_smem[];
     float* vs = reinterpret_cast<float*>(tks_smem);                     // [d]
     __shared__ unsigned hist[256];
@@ -282,6 +283,7 @@ tk_small_kernel(const float* __restrict__ a, i64 pitch_a, const float* b, i64 pi
         if (key == T) { take = eq_before < need_ties; ++eq_before; }
         if (take) {
             io[pos] = j; vo[pos] = v; ++pos;
+            flag_nonfinite(status, v);
             if (apply_to) {            // g_i <- g_i + c_i on the selected coordinate (Algorithm 2, node loop)
                 float* p = apply_to + (i64)blockIdx.x * pitch_apply + j;
                 *p = __fadd_rn(*p, v);

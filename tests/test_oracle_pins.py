@@ -314,6 +314,47 @@ def test_theorem_1_lyapunov_descent_and_rate(oracle64):
     assert np.mean(sq_norms) <= 2 * (f0 - 0.0) / (gamma * T) + G0 / (theta * T)
 
 
+def test_diagnostics_closed_forms_at_the_origin(oracle64):
+    # Section 3.3: G^t = (1/n) sum_i ||g_i^t - grad f_i(x^t)||^2.  At x = 0 the gradient of Eq. 19 is
+    # grad f_i(0) = -A_i^T y_i / (2 m_i) (sigmoid(0) = 1/2, the regulariser's derivative vanishes), so with
+    # g_i = 0:  G = (1/n) sum_i ||A_i^T y_i||^2 / (4 m_i^2)  and  ||grad f(0)||^2 = ||(1/n) sum_i A_i^T y_i / (2 m_i)||^2.
+    # The two differ by where 1/n sits, so a dropped or misplaced 1/n in either fails here.
+    w = inputs.config(0)
+    off = w.row_offsets
+    per_worker = []
+    for i in range(w.n):
+        Ai = w.A[off[i]:off[i + 1]].astype(np.float64)
+        yi = w.y[off[i]:off[i + 1]].astype(np.float64)
+        per_worker.append(-(Ai.T @ yi) / (2.0 * (off[i + 1] - off[i])))
+    per_worker = np.array(per_worker)
+    G_expect = np.sum(per_worker ** 2) / w.n
+    nrm_expect = np.sum(np.mean(per_worker, axis=0) ** 2)
+    zeros = np.zeros((w.n, w.d))
+    nrm2, G = oracle64.diagnostics(w.A, w.y, off, np.zeros(w.d), w.lam, zeros)
+    assert G == pytest.approx(G_expect, rel=1e-13)
+    assert nrm2 == pytest.approx(nrm_expect, rel=1e-13)
+    assert G > 2 * nrm2           # heterogeneous shards: the mean of squares is not the square of the mean
+
+
+def test_diagnostics_zero_and_planted_distortion(oracle64):
+    # G = 0 exactly when every g_i is the local gradient (initialisation g_i^0 = grad f_i(x^0), Section 3.3, last
+    # paragraph); with g_i = grad f_i(x) + E_i for a planted E it is ||E||_F^2 / n whatever x is.
+    w = inputs.config(0)
+    rng = np.random.default_rng(5)
+    x = rng.standard_normal(w.d) * 0.3
+    grads = oracle64.all_grads(w.A, w.y, w.row_offsets, x, w.lam)
+    nrm2, G = oracle64.diagnostics(w.A, w.y, w.row_offsets, x, w.lam, grads)
+    assert G == 0.0
+    assert nrm2 == pytest.approx(np.sum(np.mean(grads, axis=0) ** 2), rel=1e-13)
+    E = np.zeros((w.n, w.d)); E[0, 3] = 0.5; E[2, 10] = -2.0; E[3, 63] = 1.0      # exactly representable
+    _, G = oracle64.diagnostics(w.A, w.y, w.row_offsets, x, w.lam, grads + E)
+    assert G == pytest.approx((0.25 + 4.0 + 1.0) / w.n, rel=1e-12)
+    # a state built by the oracle in mode 2 (g_i^0 = grad f_i(x^0)) starts with G^0 = 0
+    st = oracle_mod.State(oracle64, w.n, w.d, w.k, w.gamma, w.lam, w.A, w.y, w.row_offsets, w.x0)
+    st.init(2)
+    assert oracle64.diagnostics(w.A, w.y, w.row_offsets, st.x, w.lam, st.gi)[1] == 0.0
+
+
 def test_theory_constants_closed_forms():
     # Section 3.3 and Example 1: sqrt(beta/theta) = sqrt(1-alpha)/(1-sqrt(1-alpha)) = (1+sqrt(1-alpha))/alpha - 1.
     for alpha in (1 / 300, 4 / 64, 0.5, 0.999):

@@ -2,8 +2,9 @@
 afford cudaMalloc's implicit synchronisation, a plug-in in a framework that owns all device
 memory, a process with a fixed memory carve-up).  Its scratch is a fixed array inside the library,
 so the test checks, through the C ABI, that it gives exactly what ef21_topk gives with a
-caller-provided workspace, twice in a row (the shared scratch keeps the previous call's contents),
-and that sizes beyond the built-in scratch are refused.  Collected last on purpose."""
+caller-provided workspace and what the CPU oracle's full-sort Top-k gives, twice in a row (the
+shared scratch keeps the previous call's contents), and that sizes beyond the built-in scratch
+are refused.  Collected last on purpose."""
 import numpy as np
 import pytest
 import torch
@@ -13,7 +14,7 @@ import ef21_inputs as inputs
 pytestmark = pytest.mark.gpu
 
 
-def test_topk_static_matches_topk_twice_in_a_row():
+def test_topk_static_matches_topk_twice_in_a_row(oracle32):
     from paper_2106_05203_b200 import binding as B
     rng = np.random.default_rng(11)
     first = np.stack([inputs.stress_vector(21, i, 100003) for i in range(7)])
@@ -28,6 +29,10 @@ def test_topk_static_matches_topk_twice_in_a_row():
         torch.cuda.synchronize()
         assert torch.equal(idx, want_idx)
         assert torch.equal(val.view(torch.int32), want_val.view(torch.int32))
+        for i in range(V.shape[0]):
+            oi, ov = oracle32.topk(V[i], k)
+            np.testing.assert_array_equal(idx[i].cpu().numpy(), oi)
+            np.testing.assert_array_equal(val[i].cpu().numpy().view(np.uint32), ov.view(np.uint32))
 
 
 def test_topk_static_refuses_sizes_beyond_its_scratch():
