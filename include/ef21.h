@@ -293,6 +293,15 @@ ef21_status ef21_get_persistent_shape(const ef21_ctx* ctx, int32_t* cluster_bloc
 ef21_status ef21_set_persistent_threads(ef21_ctx* ctx, int32_t threads_per_block);
 int32_t ef21_get_persistent_threads(const ef21_ctx* ctx);
 
+/* Body of the persistent kernel: 0 = automatic, 1 = one warp of every block serves it (adds the warps' partials,
+ * and in the leader forms the gradient, selects by warp arg-max rounds; every block's serving warp gathers the
+ * messages and updates g and x) while the other warps only sweep rows and never meet a block-wide barrier;
+ * k <= 8, Algorithms 2 and 4.  2 = every step is taken by the whole block between block barriers (any k <= 32;
+ * the only body of Algorithm 3).  Both give the same bits.  A forced body that cannot run the shape behaves as
+ * in ef21_set_persistent_shape.  get_ reports what the last persistent launch used. */
+ef21_status ef21_set_persistent_body(ef21_ctx* ctx, int32_t body);
+int32_t ef21_get_persistent_body(const ef21_ctx* ctx);
+
 /* Forces an execution path (EF21_PATH_*) for later ef21_step calls. */
 ef21_status ef21_set_path(ef21_ctx* ctx, int32_t path);
 /* The path the last ef21_step / ef21_step_grads actually used (EF21_PATH_*), 0 if none yet. */

@@ -58,6 +58,8 @@ SIGNATURES = {
     "ef21_clear_status": (ctypes.c_int, [_vp]),
     "ef21_selftest_bounded_wait": (ctypes.c_int, [_vp, ctypes.c_uint32]),
     "ef21_selftest_exchange_floor": (ctypes.c_int, [_vp, ctypes.c_int32]),
+    "ef21_set_persistent_body": (ctypes.c_int, [_vp, ctypes.c_int32]),
+    "ef21_get_persistent_body": (ctypes.c_int32, [_vp]),
     "ef21_set_persistent_shape": (ctypes.c_int, [_vp, _i32, _i32, _i32]),
     "ef21_get_persistent_shape": (ctypes.c_int, [_vp, ctypes.POINTER(_i32), ctypes.POINTER(_i32), ctypes.POINTER(_i32)]),
     "ef21_set_persistent_threads": (ctypes.c_int, [_vp, _i32]),
@@ -269,6 +271,12 @@ class EF21:
 
     def selftest_bounded_wait(self, spin_limit: int) -> None:
         _check(_lib.ef21_selftest_bounded_wait(self._h, spin_limit), "ef21_selftest_bounded_wait")
+
+    def set_persistent_body(self, body: int) -> None:
+        _check(_lib.ef21_set_persistent_body(self._h, body), "ef21_set_persistent_body")
+
+    def get_persistent_body(self) -> int:
+        return int(_lib.ef21_get_persistent_body(self._h))
 
     def selftest_exchange_floor(self, steps: int) -> None:
         _check(_lib.ef21_selftest_exchange_floor(self._h, steps), "ef21_selftest_exchange_floor")

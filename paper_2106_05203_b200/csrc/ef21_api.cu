@@ -170,6 +170,7 @@ struct ef21_ctx {
     bool agg_off_static;                // one tile only: the offsets are (0, k) whatever the messages; written once
     int pk_cluster, pk_rb, pk_src, pk_threads;      // forced persistent-kernel shape (0 / -1 = automatic)
     int pk_used_cluster, pk_used_rb, pk_used_src, pk_used_threads;
+    int pk_body, pk_used_body;          // persistent kernel body: 0 automatic, 1 compute warps + service warp, 2 whole-block steps
     unsigned spin_limit;
     bool force_general_topk;
     int variant;                        // EF21_VARIANT_*
@@ -550,6 +551,7 @@ ef21_status finish_load(ef21_ctx* c, const i64* row_offsets_host) {
 
 struct PersistPlan {
     bool ok;
+    bool roles;         // persistent_roles.inc (the last warp serves the block) instead of whole-block steps
     int C, rb, src, chunks, threads, extra;
     size_t smem;
     PersistKernel kernel;
@@ -567,10 +569,34 @@ size_t pk_smem_bytes(bool plus, int n, int k, int ld, int C, int nmsg, int src, 
     return b;
 }
 
-// Chooses cluster size, block size, rows per batch and the source of the shard rows; checks that all n
-// clusters can be resident at once (the blocks wait on one another through global memory).
+// Shared memory of the kernel whose last warp serves the block (persistent_roles.inc): x, g, g_i, message
+// sums, one partial per compute warp, the partials of the cluster's blocks, the message flags, the row slice.
+size_t pk_roles_smem_bytes(int ld, int C, int src, i64 rows_cta, int threads) {
+    size_t b = (size_t)(6 + threads / 32 + C) * ld * 4 + (size_t)((ld + 15) & ~15);
+    if (src == PK_SRC_SMEM) b += (size_t)rows_cta * ld * 4;
+    return b;
+}
+
+PersistPlan plan_persistent_body(ef21_ctx* c, bool floor_only, bool roles);
+
+// Chooses the kernel body, cluster size, block size, rows per batch and the source of the shard rows; checks
+// that all n clusters can be resident at once (the blocks wait on one another through global memory).
 PersistPlan plan_persistent(ef21_ctx* c, bool floor_only = false) {
-    PersistPlan P; P.ok = false;
+    // Automatic choice: the serving-warp body for Top-1 (2.8 against 3.0 us per iteration on the mushrooms-shaped
+    // workload, 3.7 against 4.6 on the a9a-shaped one, 10.0 against 10.4 on the w8a-shaped one, measured); with more
+    // entries per message its k arg-max rounds in one warp cost more than the whole block counting ranks.
+    const bool roles_can = c->variant != EF21_VARIANT_EF21_PLUS && c->k <= PK_ROLES_MAX_K;
+    const bool roles_first = c->pk_body == 1 || (c->pk_body == 0 && c->k == 1);
+    if (roles_can && roles_first) {
+        PersistPlan P = plan_persistent_body(c, floor_only, true);
+        if (P.ok || c->pk_body == 1) return P;
+    }
+    if (c->pk_body == 1) { PersistPlan P; P.ok = false; return P; }
+    return plan_persistent_body(c, floor_only, false);
+}
+
+PersistPlan plan_persistent_body(ef21_ctx* c, bool floor_only, bool roles) {
+    PersistPlan P; P.ok = false; P.roles = roles;
     const int ld = (int)c->L.ld;
     if (!c->shards_loaded || ld > 512 || c->k > PK_MAX_K || (i64)c->n * c->k > PK_MAX_MSGS) return P;
     const bool plus = c->variant == EF21_VARIANT_EF21_PLUS;
@@ -601,7 +627,9 @@ PersistPlan plan_persistent(ef21_ctx* c, bool floor_only = false) {
         }
         if (!rb) {
             rb = max_rb512; threads = 512;
-            src = pk_smem_bytes(plus, c->n, c->k, ld, C, nmsg, PK_SRC_SMEM, rows_cta, threads) <= (size_t)max_smem - 1024 ? PK_SRC_SMEM : PK_SRC_GMEM;
+            const size_t with_slice = roles ? pk_roles_smem_bytes(ld, C, PK_SRC_SMEM, rows_cta, threads)
+                                            : pk_smem_bytes(plus, c->n, c->k, ld, C, nmsg, PK_SRC_SMEM, rows_cta, threads);
+            src = with_slice <= (size_t)max_smem - 1024 ? PK_SRC_SMEM : PK_SRC_GMEM;
         }
         if (c->pk_threads > 0) {
             threads = c->pk_threads;
@@ -641,19 +669,27 @@ PersistPlan plan_persistent(ef21_ctx* c, bool floor_only = false) {
         const i64 rows_cta = shape_for(C, rb, src, threads, extra);
         if (c->pk_cluster == 0 && C > 1 && rows_cta < 8) continue;       // do not split below one batch
         if (src == PK_SRC_REG && ceil_div(rows_cta, rb + extra) > threads / 32) continue;
-        const size_t smem = pk_smem_bytes(plus, c->n, c->k, ld, C, nmsg, src, rows_cta, threads);
+        const size_t smem = roles ? pk_roles_smem_bytes(ld, C, src, rows_cta, threads)
+                                  : pk_smem_bytes(plus, c->n, c->k, ld, C, nmsg, src, rows_cta, threads);
         if (smem > (size_t)max_smem - 1024) continue;
-        PersistKernel kern = floor_only ? pk_lookup_floor(chunk_slots, rb, src, threads, extra)
-                             : c->variant == EF21_VARIANT_EF ? pk_lookup_ef(chunk_slots, rb, src, threads, extra)
-                             : (plus ? pk_lookup_plus(chunk_slots, rb, src, threads, extra)
-                                     : pk_lookup_ef21(chunk_slots, rb, src, threads, extra));
+        PersistKernel kern;
+        if (roles)
+            kern = floor_only ? pk_lookup_floor(chunk_slots, rb, src, threads, extra)
+                   : c->variant == EF21_VARIANT_EF ? pk_lookup_ef(chunk_slots, rb, src, threads, extra)
+                                                   : pk_lookup_ef21(chunk_slots, rb, src, threads, extra);
+        else
+            kern = floor_only ? pk_lookup_wide_floor(chunk_slots, rb, src, threads, extra)
+                   : c->variant == EF21_VARIANT_EF ? pk_lookup_wide_ef(chunk_slots, rb, src, threads, extra)
+                   : (plus ? pk_lookup_plus(chunk_slots, rb, src, threads, extra)
+                           : pk_lookup_wide_ef21(chunk_slots, rb, src, threads, extra));
         if (!kern) continue;
+        const int block_threads = threads;
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
             cudaGetLastError();
             continue;
         }
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)(c->n * C)); cfg.blockDim = dim3((unsigned)threads); cfg.dynamicSmemBytes = smem;
+        cfg.gridDim = dim3((unsigned)(c->n * C)); cfg.blockDim = dim3((unsigned)block_threads); cfg.dynamicSmemBytes = smem;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = (unsigned)C; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
@@ -679,7 +715,8 @@ ef21_status run_persistent(ef21_ctx* c, const PersistPlan& P, int steps) {
     p.spin_limit = c->spin_limit; p.epoch0 = 0u;
     CU(cudaMemsetAsync(p.slots, 0, (size_t)2 * c->n * c->k * 8, c->stream));
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(c->n * P.C)); cfg.blockDim = dim3((unsigned)P.threads); cfg.dynamicSmemBytes = P.smem;
+    cfg.gridDim = dim3((unsigned)(c->n * P.C)); cfg.blockDim = dim3((unsigned)P.threads);
+    cfg.dynamicSmemBytes = P.smem;
     cfg.stream = c->stream;
     // A plain cluster launch: that all n clusters fit on the device at once was checked with the
     // occupancy query when the plan was made.
@@ -691,6 +728,7 @@ ef21_status run_persistent(ef21_ctx* c, const PersistPlan& P, int steps) {
     if (e != cudaSuccess) { cudaGetLastError(); return EF21_ERR_CUDA; }
     c->launches += 1;
     c->pk_used_cluster = P.C; c->pk_used_rb = P.rb; c->pk_used_src = P.src; c->pk_used_threads = P.threads;
+    c->pk_used_body = P.roles ? 1 : 2;
     return EF21_OK;
 }
 
@@ -738,6 +776,7 @@ ef21_status ef21_create(ef21_ctx** out, int32_t n, int64_t d, int32_t k, float g
     c->path = EF21_PATH_AUTO; c->last_path = 0; c->launches = 0;
     c->pk_cluster = 0; c->pk_rb = 0; c->pk_src = -1; c->pk_threads = 0; c->agg_off_ready = false; c->agg_off_static = false;
     c->pk_used_cluster = c->pk_used_rb = 0; c->pk_used_src = -1; c->pk_used_threads = 0;
+    c->pk_body = 0; c->pk_used_body = 0;
     c->spin_limit = 1u << 22;
     c->force_general_topk = false;
     c->variant = EF21_VARIANT_EF21;
@@ -1123,6 +1162,14 @@ ef21_status ef21_set_persistent_threads(ef21_ctx* c, int32_t threads_per_block) 
 }
 
 int32_t ef21_get_persistent_threads(const ef21_ctx* c) { return c ? c->pk_used_threads : 0; }
+
+ef21_status ef21_set_persistent_body(ef21_ctx* c, int32_t body) {
+    if (!c || body < 0 || body > 2) return EF21_ERR_INVALID_ARG;
+    c->pk_body = body;
+    return EF21_OK;
+}
+
+int32_t ef21_get_persistent_body(const ef21_ctx* c) { return c ? c->pk_used_body : 0; }
 
 ef21_status ef21_get_persistent_shape(const ef21_ctx* c, int32_t* cluster_blocks, int32_t* rows_per_batch, int32_t* row_source) {
     if (!c) return EF21_ERR_INVALID_ARG;

@@ -113,6 +113,21 @@ __device__ __forceinline__ void st_async_f4(unsigned remote_dst, float4 v, unsig
                  ::"r"(remote_dst), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "r"(remote_bar) : "memory");
 }
 
+// Named barriers of a block (id 1..15; 0 belongs to __syncthreads): `count` threads take part, some only announce
+// their arrival (producers), the others wait for everybody (consumers).  Shared-memory writes made before the
+// arrival are visible to the threads the barrier releases.
+__device__ __forceinline__ void named_bar_sync(int id, int count) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+__device__ __forceinline__ void named_bar_arrive(int id, int count) {
+    asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+
+// Keeps the compiler from moving loads and stores from one phase of an iteration into another.  The service warp of
+// the persistent kernel runs alone, so the order of its instructions is its timing: with the phases kept apart the
+// iteration was 8-18 % shorter than with the order the compiler chose on its own (measured, both orders correct).
+__device__ __forceinline__ void phase_fence() { asm volatile("" ::: "memory"); }
+
 __device__ __forceinline__ float comp_of(const float4& v, int c) {
     return c == 0 ? v.x : (c == 1 ? v.y : (c == 2 ? v.z : v.w));
 }
@@ -122,9 +137,17 @@ typedef void (*PersistKernel)(const PersistParams);
 // One lookup per method (each in a translation unit of its own, so that they compile side by side):
 // the kernel instantiated for (chunk slots per lane, rows per warp batch, row source, threads per block,
 // extra rows per batch), or nullptr if that shape is not instantiated.
-PersistKernel pk_lookup_ef21(int chunks, int rb, int src, int threads, int extra);     // Algorithm 2
-PersistKernel pk_lookup_plus(int chunks, int rb, int src, int threads, int extra);     // Algorithm 3
-PersistKernel pk_lookup_ef(int chunks, int rb, int src, int threads, int extra);       // Algorithm 4
-PersistKernel pk_lookup_floor(int chunks, int rb, int src, int threads, int extra);    // exchange skeleton (measuring aid)
+// Two bodies exist.  "roles" (persistent_roles.inc): the last warp of a block serves it, the others only sweep rows;
+// Top-k by warp arg-max rounds -- for k <= PK_ROLES_MAX_K.  "wide" (persistent_body.inc): every step is taken by the
+// whole block between block barriers, Top-k by rank counting over all threads for larger k -- any k <= PK_MAX_K, and
+// the only body of Algorithm 3.
+constexpr int PK_ROLES_MAX_K = 8;
+PersistKernel pk_lookup_ef21(int chunks, int rb, int src, int threads, int extra);          // Algorithm 2, roles
+PersistKernel pk_lookup_ef(int chunks, int rb, int src, int threads, int extra);            // Algorithm 4, roles
+PersistKernel pk_lookup_floor(int chunks, int rb, int src, int threads, int extra);         // exchange skeleton, roles
+PersistKernel pk_lookup_wide_ef21(int chunks, int rb, int src, int threads, int extra);     // Algorithm 2, wide
+PersistKernel pk_lookup_plus(int chunks, int rb, int src, int threads, int extra);          // Algorithm 3, wide
+PersistKernel pk_lookup_wide_ef(int chunks, int rb, int src, int threads, int extra);       // Algorithm 4, wide
+PersistKernel pk_lookup_wide_floor(int chunks, int rb, int src, int threads, int extra);    // exchange skeleton, wide
 
 }  // namespace ef21

@@ -1,4 +1,5 @@
-// Persistent cluster kernel for EF21 (Algorithm 2): instantiations and their lookup.
+// Persistent cluster kernel for EF21 (Algorithm 2), compute warps + service warp: instantiations and their lookup.
+#define PK_BODY_FILE "persistent_roles.inc"
 #define PK_KERNEL_NAME persistent_kernel
 #define PK_LOOKUP_NAME pk_lookup_ef21
 #define PK_PLUS 0

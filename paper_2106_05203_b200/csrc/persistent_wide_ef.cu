@@ -1,0 +1,8 @@
+// Persistent cluster kernel for the original error feedback method (Algorithm 4), whole-block steps (larger k).
+#define PK_BODY_FILE "persistent_body.inc"
+#define PK_KERNEL_NAME persistent_wide_ef_kernel
+#define PK_LOOKUP_NAME pk_lookup_wide_ef
+#define PK_PLUS 0
+#define PK_EF 1
+#define PK_FLOOR 0
+#include "persistent_method.inc"

@@ -426,6 +426,43 @@ def test_persistent_block_sizes(d, rb, threads, src, B, oracle32):
     assert h.poll() == 0
 
 
+@pytest.mark.parametrize("body", [1, 2], ids=["serving-warp", "whole-block"])
+@pytest.mark.parametrize("cfg,k,steps", [(0, 4, 30), (0, 1, 30), (1, 1, 60), (2, 4, 20), (3, 1, 15)])
+def test_persistent_bodies_track_the_oracle(cfg, k, steps, body, B, oracle32):
+    # both bodies of the persistent kernel on every kind of shape (rows in registers, one extra row per warp, rows
+    # from global memory; one and several polling rounds), iteration by iteration against the oracle
+    w = inputs.config(cfg, k=k)
+    h = make_gpu(w, k=k, path=2); h.set_persistent_body(body)
+    st = make_oracle_state(oracle32, w, k=k)
+    h.init(0); st.init(0)
+    lockstep(h, st, oracle32, w, steps, k=k)
+    assert h.last_path == B.PATH_PERSISTENT and h.get_persistent_body() == body
+    # several iterations in one launch give the same bits as the same iterations one launch each
+    outs = []
+    for chunks in ((7,), (1,) * 7):
+        h2 = make_gpu(w, k=k, path=2); h2.set_persistent_body(body); h2.init(0)
+        for s_ in chunks:
+            h2.step(s_)
+        outs.append(h2.get_state_host())
+    for a_, b_ in zip(outs[0], outs[1]):
+        np.testing.assert_array_equal(a_, b_)
+    assert h.poll() == 0 and h2.poll() == 0
+
+
+def test_persistent_body_choice(B):
+    w = inputs.config(0, k=1)
+    h = make_gpu(w, k=1, path=2); h.init(0); h.step(2)
+    assert h.get_persistent_body() == 1                 # Top-1: the serving-warp body
+    w = inputs.config(0, k=4)
+    h = make_gpu(w, k=4, path=2); h.init(0); h.step(2)
+    assert h.get_persistent_body() == 2                 # several entries per message: whole-block steps
+    w = inputs.config(0, k=16)
+    h = make_gpu(w, k=16, path=2); h.set_persistent_body(1); h.init(0)
+    with pytest.raises(B.Ef21Error) as e:
+        h.step(1)                                       # the serving-warp body stops at k = 8
+    assert e.value.status == 7
+
+
 def test_persistent_many_steps_in_one_launch_equals_single_steps(B):
     w = inputs.config(1)
     a = make_gpu(w, path=2); a.init(0); a.step(300)
