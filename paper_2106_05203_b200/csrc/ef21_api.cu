@@ -158,6 +158,15 @@ bool valid_shape(i64 n, i64 d, i64 k, i64 N) {
 
 }  // namespace
 
+// Launch plan of the persistent path (made by plan_persistent, kept in the handle until something it depends on changes).
+struct PersistPlan {
+    bool ok;
+    bool roles;         // persistent_roles.inc (the last warp serves the block) instead of whole-block steps
+    int C, rb, src, chunks, threads, extra;
+    size_t smem;
+    PersistKernel kernel;
+};
+
 struct ef21_ctx {
     int n; i64 d; int k; float gamma, lambda; i64 N;
     cudaStream_t stream;
@@ -170,6 +179,8 @@ struct ef21_ctx {
     bool agg_off_static;                // one tile only: the offsets are (0, k) whatever the messages; written once
     int pk_cluster, pk_rb, pk_src, pk_threads;      // forced persistent-kernel shape (0 / -1 = automatic)
     int pk_used_cluster, pk_used_rb, pk_used_src, pk_used_threads;
+    PersistPlan plan; bool plan_valid;  // cached plan of ef21_step's persistent launch
+    unsigned pk_epoch, pk_par;          // epoch and slot half of the last persistent iteration (see PersistParams)
     int pk_body, pk_used_body;          // persistent kernel body: 0 automatic, 1 compute warps + service warp, 2 whole-block steps
     unsigned spin_limit;
     bool force_general_topk;
@@ -535,6 +546,7 @@ ef21_status finish_load(ef21_ctx* c, const i64* row_offsets_host) {
     if ((i64)c->num_tiles > c->L.max_tiles) return EF21_ERR_WORKSPACE;
     // a captured launch-path iteration has the old tile count baked into its grid
     if (c->iter_graph) { cudaGraphExecDestroy(c->iter_graph); c->iter_graph = nullptr; }
+    c->plan_valid = false;
     CU(cudaMemcpyAsync(c->at<i64>(c->L.row_off), c->row_off.data(), (size_t)(c->n + 1) * 8, cudaMemcpyHostToDevice, c->stream));
     CU(cudaMemcpyAsync(c->at<int>(c->L.tile_begin), c->tile_begin.data(), (size_t)(c->n + 1) * 4, cudaMemcpyHostToDevice, c->stream));
     if (c->num_tiles > 0)
@@ -549,13 +561,6 @@ ef21_status finish_load(ef21_ctx* c, const i64* row_offsets_host) {
 // Persistent path
 // ---------------------------------------------------------------------------------------------
 
-struct PersistPlan {
-    bool ok;
-    bool roles;         // persistent_roles.inc (the last warp serves the block) instead of whole-block steps
-    int C, rb, src, chunks, threads, extra;
-    size_t smem;
-    PersistKernel kernel;
-};
 
 // From two entries per worker on, the received messages are scattered into a [n][ld] table in shared
 // memory (if that table is small): aggregation then costs n reads per coordinate instead of n*k.
@@ -684,7 +689,9 @@ PersistPlan plan_persistent_body(ef21_ctx* c, bool floor_only, bool roles) {
                            : pk_lookup_wide_ef21(chunk_slots, rb, src, threads, extra));
         if (!kern) continue;
         const int block_threads = threads;
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+        // the device's opt-in limit (less the kernel's static part), so that no other handle's plan for the same
+        // kernel can lower it under this one's need
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem - 1024) != cudaSuccess) {
             cudaGetLastError();
             continue;
         }
@@ -712,8 +719,8 @@ ef21_status run_persistent(ef21_ctx* c, const PersistPlan& P, int steps) {
     p.n = c->n; p.d = (int)c->d; p.ld = (int)c->L.ld; p.k = c->k; p.C = P.C; p.steps = steps;
     p.objective = c->objective;
     p.slice_rows = 0; p.use_table = (c->variant != EF21_VARIANT_EF21_PLUS && pk_use_table(c->n, (int)c->L.ld, c->k)) ? 1 : 0; p.gamma = c->gamma; p.lambda = c->lambda; p.inv_n = 1.0f / (float)c->n;
-    p.spin_limit = c->spin_limit; p.epoch0 = 0u;
-    CU(cudaMemsetAsync(p.slots, 0, (size_t)2 * c->n * c->k * 8, c->stream));
+    // the epochs run on from launch to launch, so the slot array (cleared once, at creation) needs no clearing here
+    p.spin_limit = c->spin_limit; p.epoch0 = c->pk_epoch; p.par0 = c->pk_par;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(c->n * P.C)); cfg.blockDim = dim3((unsigned)P.threads);
     cfg.dynamicSmemBytes = P.smem;
@@ -727,6 +734,8 @@ ef21_status run_persistent(ef21_ctx* c, const PersistPlan& P, int steps) {
     cudaError_t e = cudaLaunchKernelEx(&cfg, P.kernel, p);
     if (e != cudaSuccess) { cudaGetLastError(); return EF21_ERR_CUDA; }
     c->launches += 1;
+    c->pk_epoch = (unsigned)(((i64)c->pk_epoch + steps - 1) % 65535) + 1u;
+    c->pk_par = (c->pk_par + (unsigned)steps) & 1u;
     c->pk_used_cluster = P.C; c->pk_used_rb = P.rb; c->pk_used_src = P.src; c->pk_used_threads = P.threads;
     c->pk_used_body = P.roles ? 1 : 2;
     return EF21_OK;
@@ -776,7 +785,7 @@ ef21_status ef21_create(ef21_ctx** out, int32_t n, int64_t d, int32_t k, float g
     c->path = EF21_PATH_AUTO; c->last_path = 0; c->launches = 0;
     c->pk_cluster = 0; c->pk_rb = 0; c->pk_src = -1; c->pk_threads = 0; c->agg_off_ready = false; c->agg_off_static = false;
     c->pk_used_cluster = c->pk_used_rb = 0; c->pk_used_src = -1; c->pk_used_threads = 0;
-    c->pk_body = 0; c->pk_used_body = 0;
+    c->pk_body = 0; c->pk_used_body = 0; c->pk_epoch = 0u; c->pk_par = 0u; c->plan_valid = false;
     c->spin_limit = 1u << 22;
     c->force_general_topk = false;
     c->variant = EF21_VARIANT_EF21;
@@ -791,6 +800,7 @@ ef21_status ef21_create(ef21_ctx** out, int32_t n, int64_t d, int32_t k, float g
     if (e == cudaSuccess) e = cudaMemsetAsync(c->msg_val(), 0, (size_t)n * k * 4, c->stream);
     if (e == cudaSuccess && L.tk.fast) e = cudaMemsetAsync(c->ws + L.topk + L.tk.slow_count, 0, 4, c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->ws + L.plus_choice, 0, (size_t)n * 4, c->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->ws + L.slots, 0, (size_t)2 * n * k * 8, c->stream);
     if (e != cudaSuccess) { delete c; return EF21_ERR_CUDA; }
     *out = c;
     return EF21_OK;
@@ -926,7 +936,10 @@ ef21_status ef21_step(ef21_ctx* c, int32_t steps) {
     if (!c->shards_loaded || !c->inited) return EF21_ERR_STATE;
     if (steps == 0) return EF21_OK;
     if (c->path != EF21_PATH_LAUNCHES) {
-        PersistPlan P = plan_persistent(c);
+        // planning asks the runtime several questions (attributes, occupancy of the cluster launch): once per
+        // handle and setting, not once per call
+        if (!c->plan_valid) { c->plan = plan_persistent(c); c->plan_valid = true; }
+        const PersistPlan& P = c->plan;
         if (P.ok) {
             EF(run_persistent(c, P, steps));
             c->last_path = EF21_PATH_PERSISTENT;
@@ -1152,12 +1165,14 @@ ef21_status ef21_set_persistent_shape(ef21_ctx* c, int32_t cluster_blocks, int32
     if (rows_per_batch != 0 && rows_per_batch != 4 && rows_per_batch != 8 && rows_per_batch != 16 && rows_per_batch != 32) return EF21_ERR_INVALID_ARG;
     if (row_source < -1 || row_source > 2) return EF21_ERR_INVALID_ARG;
     c->pk_cluster = cluster_blocks; c->pk_rb = rows_per_batch; c->pk_src = row_source;
+    c->plan_valid = false;
     return EF21_OK;
 }
 
 ef21_status ef21_set_persistent_threads(ef21_ctx* c, int32_t threads_per_block) {
     if (!c || (threads_per_block != 0 && threads_per_block != 256 && threads_per_block != 512)) return EF21_ERR_INVALID_ARG;
     c->pk_threads = threads_per_block;
+    c->plan_valid = false;
     return EF21_OK;
 }
 
@@ -1166,6 +1181,7 @@ int32_t ef21_get_persistent_threads(const ef21_ctx* c) { return c ? c->pk_used_t
 ef21_status ef21_set_persistent_body(ef21_ctx* c, int32_t body) {
     if (!c || body < 0 || body > 2) return EF21_ERR_INVALID_ARG;
     c->pk_body = body;
+    c->plan_valid = false;
     return EF21_OK;
 }
 
@@ -1188,6 +1204,7 @@ ef21_status ef21_set_objective(ef21_ctx* c, int32_t objective) {
 ef21_status ef21_set_variant(ef21_ctx* c, int32_t variant) {
     if (!c || variant < EF21_VARIANT_EF21 || variant > EF21_VARIANT_EF) return EF21_ERR_INVALID_ARG;
     c->variant = variant;
+    c->plan_valid = false;
     return EF21_OK;
 }
 

@@ -64,7 +64,8 @@ struct PersistParams {
     int use_table;             // 1: received messages are scattered into a [n][ld] table in shared memory
     float gamma, lambda, inv_n;
     unsigned spin_limit;
-    unsigned epoch0;           // epoch of the first iteration minus one
+    unsigned epoch0;           // epoch of the handle's last iteration so far (0: none yet); epochs run 1..65535 and wrap to 1
+    unsigned par0;             // which half of the slot array that iteration used
     int* plus_choice;          // [n] EF21+: branch taken at the final iteration (0 Markov compressor, 1 plain)
 };
 
@@ -131,6 +132,10 @@ __device__ __forceinline__ void phase_fence() { asm volatile("" ::: "memory"); }
 __device__ __forceinline__ float comp_of(const float4& v, int c) {
     return c == 0 ? v.x : (c == 1 ? v.y : (c == 2 ? v.z : v.w));
 }
+
+// The epoch after e.  A slot word is at most two iterations old when it is polled, so a wrapped epoch never meets
+// its own value; 0 marks a word that no iteration has written (the array is cleared once, at creation).
+__device__ __forceinline__ unsigned next_epoch(unsigned e) { return e >= 65535u ? 1u : e + 1u; }
 
 typedef void (*PersistKernel)(const PersistParams);
 
