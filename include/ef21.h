@@ -143,12 +143,16 @@ ef21_status ef21_step(ef21_ctx* ctx, int32_t steps);
  * work ends), so a later operation on the handle's stream still sees the complete result. */
 ef21_status ef21_step_grads(ef21_ctx* ctx, const float* V_dev, int32_t steps);
 
-/* One iteration of the stochastic variant (Appendix, Algorithm 5): the loop of Algorithm 2 with
- * grad f_i(x^{t+1}) replaced by the minibatch estimate over the tau rows batch_dev[i][0..tau) of worker i's
- * shard (row numbers inside the shard, int32, leading dimension tau; the caller draws them, e.g. without
- * replacement), averaged over tau, plus the regulariser term.  Every shard needs at least tau rows.  An
- * index outside its shard is replaced by row 0 and EF21_ERR_INVALID_ARG is recorded in the status word
- * (ef21_poll).  Launch path; EF21_VARIANT_EF21 only. */
+/* `steps` iterations of the stochastic variant (Appendix, Algorithm 5): the loop of Algorithm 2 with
+ * grad f_i(x^{t+1}) replaced by the minibatch estimate over tau rows of worker i's shard, averaged over tau,
+ * plus the regulariser term.  batches_dev[steps][n][tau] holds, for every iteration and worker, the row
+ * numbers inside the shard (int32; the caller draws them, e.g. without replacement); it must stay valid until
+ * the stream has passed the call.  Every shard needs at least tau rows.  An index outside its shard is
+ * replaced by row 0 and EF21_ERR_INVALID_ARG is recorded in the status word (ef21_poll).  EF21_VARIANT_EF21
+ * only.  Shapes the persistent path takes (d <= 512, k <= 8) run all iterations in one launch, the sampled rows
+ * read from global memory each iteration; others run launch by launch.  ef21_step_minibatch is the same call
+ * for one iteration. */
+ef21_status ef21_step_minibatches(ef21_ctx* ctx, const int32_t* batches_dev, int32_t tau, int32_t steps);
 ef21_status ef21_step_minibatch(ef21_ctx* ctx, const int32_t* batch_dev, int32_t tau);
 
 /* grad f_i(x) for the current x and all workers, written to grads_out_dev[n][d]

@@ -41,6 +41,7 @@ SIGNATURES = {
     "ef21_step": (ctypes.c_int, [_vp, _i32]),
     "ef21_step_grads": (ctypes.c_int, [_vp, _vp, _i32]),
     "ef21_step_minibatch": (ctypes.c_int, [_vp, _vp, _i32]),
+    "ef21_step_minibatches": (ctypes.c_int, [_vp, _vp, _i32, _i32]),
     "ef21_local_grads": (ctypes.c_int, [_vp, _vp]),
     "ef21_topk_workspace_bytes": (_sz, [_i32, _i64, _i32]),
     "ef21_topk": (ctypes.c_int, [_vp, _i32, _i64, _i32, _vp, _vp, _vp, _sz, _vp]),
@@ -203,6 +204,15 @@ class EF21:
             raise TypeError("batch must be a contiguous int32 CUDA tensor of shape [n, tau]")
         _check(_lib.ef21_step_minibatch(self._h, _ptr(batch), int(batch.shape[1])), "ef21_step_minibatch")
         self._keep_batch = batch
+
+    def step_minibatches(self, batches: torch.Tensor) -> None:
+        """batches[steps, n, tau] int32 row numbers inside each worker's shard: that many stochastic iterations."""
+        if not (batches.is_cuda and batches.dtype == torch.int32 and batches.is_contiguous() and batches.dim() == 3
+                and batches.shape[1] == self.n):
+            raise TypeError("batches must be a contiguous int32 CUDA tensor of shape [steps, n, tau]")
+        _check(_lib.ef21_step_minibatches(self._h, _ptr(batches), int(batches.shape[2]), int(batches.shape[0])),
+               "ef21_step_minibatches")
+        self._keep_batch = batches
 
     def local_grads(self) -> torch.Tensor:
         out = torch.empty((self.n, self.d), dtype=torch.float32, device=self.device)

@@ -180,6 +180,7 @@ struct ef21_ctx {
     int pk_cluster, pk_rb, pk_src, pk_threads;      // forced persistent-kernel shape (0 / -1 = automatic)
     int pk_used_cluster, pk_used_rb, pk_used_src, pk_used_threads;
     PersistPlan plan; bool plan_valid;  // cached plan of ef21_step's persistent launch
+    PersistPlan mb_plan; bool mb_plan_valid; int mb_plan_tau;      // the same for the stochastic variant with mb_plan_tau rows
     unsigned pk_epoch, pk_par;          // epoch and slot half of the last persistent iteration (see PersistParams)
     int pk_body, pk_used_body;          // persistent kernel body: 0 automatic, 1 compute warps + service warp, 2 whole-block steps
     unsigned spin_limit;
@@ -546,7 +547,7 @@ ef21_status finish_load(ef21_ctx* c, const i64* row_offsets_host) {
     if ((i64)c->num_tiles > c->L.max_tiles) return EF21_ERR_WORKSPACE;
     // a captured launch-path iteration has the old tile count baked into its grid
     if (c->iter_graph) { cudaGraphExecDestroy(c->iter_graph); c->iter_graph = nullptr; }
-    c->plan_valid = false;
+    c->plan_valid = false; c->mb_plan_valid = false;
     CU(cudaMemcpyAsync(c->at<i64>(c->L.row_off), c->row_off.data(), (size_t)(c->n + 1) * 8, cudaMemcpyHostToDevice, c->stream));
     CU(cudaMemcpyAsync(c->at<int>(c->L.tile_begin), c->tile_begin.data(), (size_t)(c->n + 1) * 4, cudaMemcpyHostToDevice, c->stream));
     if (c->num_tiles > 0)
@@ -582,7 +583,7 @@ size_t pk_roles_smem_bytes(int ld, int C, int src, i64 rows_cta, int threads) {
     return b;
 }
 
-PersistPlan plan_persistent_body(ef21_ctx* c, bool floor_only, bool roles);
+PersistPlan plan_persistent_body(ef21_ctx* c, bool floor_only, bool roles, int tau = 0);
 
 // Chooses the kernel body, cluster size, block size, rows per batch and the source of the shard rows; checks
 // that all n clusters can be resident at once (the blocks wait on one another through global memory).
@@ -600,7 +601,8 @@ PersistPlan plan_persistent(ef21_ctx* c, bool floor_only = false) {
     return plan_persistent_body(c, floor_only, false);
 }
 
-PersistPlan plan_persistent_body(ef21_ctx* c, bool floor_only, bool roles) {
+// tau > 0: plan for the stochastic variant (tau sampled rows per worker and iteration, read from global memory).
+PersistPlan plan_persistent_body(ef21_ctx* c, bool floor_only, bool roles, int tau) {
     PersistPlan P; P.ok = false; P.roles = roles;
     const int ld = (int)c->L.ld;
     if (!c->shards_loaded || ld > 512 || c->k > PK_MAX_K || (i64)c->n * c->k > PK_MAX_MSGS) return P;
@@ -615,6 +617,7 @@ PersistPlan plan_persistent_body(ef21_ctx* c, bool floor_only, bool roles) {
     const int max_rb512 = chunk_slots == 1 ? 16 : (chunk_slots == 2 ? 8 : 4);       // rb * chunk_slots <= 16
     i64 max_m = 0;
     for (int i = 0; i < c->n; ++i) max_m = std::max<i64>(max_m, c->row_off[i + 1] - c->row_off[i]);
+    if (tau > 0) max_m = tau;
     const int nmsg = c->n * c->k;
 
     // One candidate shape for a cluster size: rows in registers with 8 warps if they fit, else with 16
@@ -647,6 +650,7 @@ PersistPlan plan_persistent_body(ef21_ctx* c, bool floor_only, bool roles) {
             if (src == PK_SRC_REG && ceil_div(rows_cta, rb) > threads / 32) src = PK_SRC_SMEM;
         }
         if (c->pk_src >= 0) src = c->pk_src;
+        if (tau > 0) src = PK_SRC_GMEM;          // sampled rows change every iteration
         return rows_cta;
     };
 
@@ -661,7 +665,7 @@ PersistPlan plan_persistent_body(ef21_ctx* c, bool floor_only, bool roles) {
             if ((i64)c->n * C > sms) break;
             int rb, src, threads, extra;
             shape_for(C, rb, src, threads, extra);
-            if (src == PK_SRC_REG && threads == 256 && rb <= 16) pref = C;
+            if ((src == PK_SRC_REG || tau > 0) && threads == 256 && rb <= 16) pref = C;
         }
         if (pref) order[norder++] = pref;
         for (int C = 8; C >= 1; --C)
@@ -710,8 +714,9 @@ PersistPlan plan_persistent_body(ef21_ctx* c, bool floor_only, bool roles) {
     return P;
 }
 
-ef21_status run_persistent(ef21_ctx* c, const PersistPlan& P, int steps) {
+ef21_status run_persistent(ef21_ctx* c, const PersistPlan& P, int steps, const int* batch = nullptr, int tau = 0) {
     PersistParams p;
+    p.batch = batch; p.tau = tau;
     p.A = c->at<float>(c->L.A); p.y = c->at<float>(c->L.y); p.row_off = c->at<i64>(c->L.row_off);
     p.x = c->x(); p.g = c->g(); p.gi = c->gi(); p.msg_idx = c->msg_idx(); p.msg_val = c->msg_val();
     p.plus_choice = c->at<int>(c->L.plus_choice);
@@ -785,7 +790,7 @@ ef21_status ef21_create(ef21_ctx** out, int32_t n, int64_t d, int32_t k, float g
     c->path = EF21_PATH_AUTO; c->last_path = 0; c->launches = 0;
     c->pk_cluster = 0; c->pk_rb = 0; c->pk_src = -1; c->pk_threads = 0; c->agg_off_ready = false; c->agg_off_static = false;
     c->pk_used_cluster = c->pk_used_rb = 0; c->pk_used_src = -1; c->pk_used_threads = 0;
-    c->pk_body = 0; c->pk_used_body = 0; c->pk_epoch = 0u; c->pk_par = 0u; c->plan_valid = false;
+    c->pk_body = 0; c->pk_used_body = 0; c->pk_epoch = 0u; c->pk_par = 0u; c->plan_valid = false; c->mb_plan_valid = false; c->mb_plan_tau = 0;
     c->spin_limit = 1u << 22;
     c->force_general_topk = false;
     c->variant = EF21_VARIANT_EF21;
@@ -1007,17 +1012,36 @@ ef21_status ef21_step_grads(ef21_ctx* c, const float* V_dev, int32_t steps) {
     return EF21_OK;
 }
 
-ef21_status ef21_step_minibatch(ef21_ctx* c, const int32_t* batch_dev, int32_t tau) {
-    if (!c || !batch_dev || tau < 1) return EF21_ERR_INVALID_ARG;
+ef21_status ef21_step_minibatches(ef21_ctx* c, const int32_t* batches_dev, int32_t tau, int32_t steps) {
+    if (!c || !batches_dev || tau < 1 || steps < 0) return EF21_ERR_INVALID_ARG;
     if (!c->shards_loaded || !c->inited) return EF21_ERR_STATE;
     if (c->variant != EF21_VARIANT_EF21) return EF21_ERR_UNSUPPORTED;
     for (int i = 0; i < c->n; ++i)
         if (c->row_off[i + 1] - c->row_off[i] < tau) return EF21_ERR_INVALID_ARG;
-    EF(enqueue_x_update(c));
-    EF(enqueue_minibatch_grads(c, batch_dev, tau));
-    EF(enqueue_round(c, c->at<float>(c->L.grad), c->L.ld, false));
+    if (steps == 0) return EF21_OK;
+    if (c->path != EF21_PATH_LAUNCHES && c->k <= PK_ROLES_MAX_K && c->pk_body != 2) {
+        if (!c->mb_plan_valid || c->mb_plan_tau != tau) {
+            c->mb_plan = plan_persistent_body(c, false, true, tau);
+            c->mb_plan_tau = tau; c->mb_plan_valid = true;
+        }
+        if (c->mb_plan.ok) {
+            EF(run_persistent(c, c->mb_plan, steps, batches_dev, tau));
+            c->last_path = EF21_PATH_PERSISTENT;
+            return EF21_OK;
+        }
+    }
+    if (c->path == EF21_PATH_PERSISTENT) return EF21_ERR_UNSUPPORTED;
+    for (int t = 0; t < steps; ++t) {
+        EF(enqueue_x_update(c));
+        EF(enqueue_minibatch_grads(c, batches_dev + (size_t)t * c->n * tau, tau));
+        EF(enqueue_round(c, c->at<float>(c->L.grad), c->L.ld, false));
+    }
     c->last_path = EF21_PATH_LAUNCHES;
     return EF21_OK;
+}
+
+ef21_status ef21_step_minibatch(ef21_ctx* c, const int32_t* batch_dev, int32_t tau) {
+    return ef21_step_minibatches(c, batch_dev, tau, 1);
 }
 
 ef21_status ef21_local_grads(ef21_ctx* c, float* grads_out_dev) {
@@ -1165,14 +1189,14 @@ ef21_status ef21_set_persistent_shape(ef21_ctx* c, int32_t cluster_blocks, int32
     if (rows_per_batch != 0 && rows_per_batch != 4 && rows_per_batch != 8 && rows_per_batch != 16 && rows_per_batch != 32) return EF21_ERR_INVALID_ARG;
     if (row_source < -1 || row_source > 2) return EF21_ERR_INVALID_ARG;
     c->pk_cluster = cluster_blocks; c->pk_rb = rows_per_batch; c->pk_src = row_source;
-    c->plan_valid = false;
+    c->plan_valid = false; c->mb_plan_valid = false;
     return EF21_OK;
 }
 
 ef21_status ef21_set_persistent_threads(ef21_ctx* c, int32_t threads_per_block) {
     if (!c || (threads_per_block != 0 && threads_per_block != 256 && threads_per_block != 512)) return EF21_ERR_INVALID_ARG;
     c->pk_threads = threads_per_block;
-    c->plan_valid = false;
+    c->plan_valid = false; c->mb_plan_valid = false;
     return EF21_OK;
 }
 
@@ -1181,7 +1205,7 @@ int32_t ef21_get_persistent_threads(const ef21_ctx* c) { return c ? c->pk_used_t
 ef21_status ef21_set_persistent_body(ef21_ctx* c, int32_t body) {
     if (!c || body < 0 || body > 2) return EF21_ERR_INVALID_ARG;
     c->pk_body = body;
-    c->plan_valid = false;
+    c->plan_valid = false; c->mb_plan_valid = false;
     return EF21_OK;
 }
 
@@ -1204,7 +1228,7 @@ ef21_status ef21_set_objective(ef21_ctx* c, int32_t objective) {
 ef21_status ef21_set_variant(ef21_ctx* c, int32_t variant) {
     if (!c || variant < EF21_VARIANT_EF21 || variant > EF21_VARIANT_EF) return EF21_ERR_INVALID_ARG;
     c->variant = variant;
-    c->plan_valid = false;
+    c->plan_valid = false; c->mb_plan_valid = false;
     return EF21_OK;
 }
 

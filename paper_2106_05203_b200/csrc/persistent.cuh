@@ -67,6 +67,8 @@ struct PersistParams {
     unsigned epoch0;           // epoch of the handle's last iteration so far (0: none yet); epochs run 1..65535 and wrap to 1
     unsigned par0;             // which half of the slot array that iteration used
     int* plus_choice;          // [n] EF21+: branch taken at the final iteration (0 Markov compressor, 1 plain)
+    const int* batch;          // stochastic variant (Algorithm 5): [steps][n][tau] row numbers inside each shard; null: all rows
+    int tau;                   // rows per worker and iteration of the stochastic variant
 };
 
 __device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long* p) {

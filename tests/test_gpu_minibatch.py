@@ -39,10 +39,11 @@ def test_minibatch_estimates(cfg, tau, B, oracle32):
     assert h.poll() == 0
 
 
+@pytest.mark.parametrize("path", [1, 2], ids=["launches", "persistent"])
 @pytest.mark.parametrize("cfg,k,tau,steps", [(0, 4, 8, 40), (1, 1, 32, 60), (2, 4, 64, 25), (3, 8, 128, 10)])
-def test_minibatch_lockstep(cfg, k, tau, steps, B, oracle32):
+def test_minibatch_lockstep(cfg, k, tau, steps, path, B, oracle32):
     w = inputs.config(cfg)
-    h = make_gpu(w, k=k); st = make_oracle_state(oracle32, w, k=k)
+    h = make_gpu(w, k=k, path=path); st = make_oracle_state(oracle32, w, k=k)
     h.init(0); st.init(0)
     batches = {}
 
@@ -54,22 +55,54 @@ def test_minibatch_lockstep(cfg, k, tau, steps, B, oracle32):
         return _batch_grads(oracle32, w, st.x, batches[t])
 
     assert lockstep(h, st, oracle32, w, steps, k=k, advance=advance, grads_of=grads_of) <= max(2, steps // 10)
-    assert h.last_path == B.PATH_LAUNCHES
+    assert h.last_path == path
     assert rel_l2(h.get_state_host()[0], st.x) <= 1e-4
     assert h.poll() == 0
 
 
+@pytest.mark.parametrize("path", [0, 1], ids=["auto", "launches"])
+@pytest.mark.parametrize("cfg,k,tau,steps", [(1, 1, 32, 80), (0, 4, 8, 30), (3, 1, 64, 12)])
+def test_many_stochastic_iterations_in_one_call(cfg, k, tau, steps, path, B, oracle32):
+    # [steps][n][tau] row numbers, one call (one launch of the persistent kernel on the automatic path): the same bits
+    # as the same iterations one call each, and the oracle's trajectory
+    w = inputs.config(cfg)
+    all_rows = np.stack([inputs.minibatch_rows(9, t, w.row_offsets, tau) for t in range(steps)])
+    outs = []
+    for single in (False, True):
+        h = make_gpu(w, k=k, path=path); h.init(0)
+        if single:
+            for t in range(steps):
+                h.step_minibatches(dev(all_rows[t:t + 1], torch.int32))
+        else:
+            h.step_minibatches(dev(all_rows, torch.int32))
+        assert h.last_path == (B.PATH_PERSISTENT if path == 0 else B.PATH_LAUNCHES)
+        assert h.poll() == 0
+        outs.append(h.get_state_host())
+    for u, v in zip(*outs):
+        np.testing.assert_array_equal(u, v)
+    st = make_oracle_state(oracle32, w, k=k); st.init(0)
+    for t in range(steps):
+        st.step_minibatch(all_rows[t])
+    assert rel_l2(outs[0][0], st.x) <= 1e-4
+
+
 def test_full_batch_in_order_matches_the_deterministic_step(B, oracle32):
-    # tau = m_i with the identity order visits the same rows in the same tiles as the full gradient
+    # tau = m_i with the identity order visits the same rows in the same order as the full gradient: the same bits,
+    # on the launch path (same tiles) and on the persistent path (same cluster shape, rows from global memory)
     w = inputs.config(0)
     m = int(np.min(np.diff(w.row_offsets)))
-    a = make_gpu(w, path=B.PATH_LAUNCHES); b = make_gpu(w)
-    a.init(0); b.init(0)
     batch = dev(np.tile(np.arange(m, dtype=np.int32), (w.n, 1)), torch.int32)
-    for _ in range(10):
-        a.step(1); b.step_minibatch(batch)
-    for u, v in zip(a.get_state_host(), b.get_state_host()):
-        np.testing.assert_array_equal(u, v)
+    for path in (B.PATH_LAUNCHES, B.PATH_PERSISTENT):
+        a = make_gpu(w, k=1, path=path); b = make_gpu(w, k=1, path=path)
+        if path == B.PATH_PERSISTENT:
+            for h in (a, b):
+                h.set_persistent_shape(2, 8, 2); h.set_persistent_threads(256)
+        a.init(0); b.init(0)
+        for _ in range(10):
+            a.step(1); b.step_minibatch(batch)
+        assert a.last_path == path and b.last_path == path
+        for u, v in zip(a.get_state_host(), b.get_state_host()):
+            np.testing.assert_array_equal(u, v)
 
 
 def test_changing_tau_rebuilds_the_tile_table(B, oracle32):
@@ -83,9 +116,10 @@ def test_changing_tau_rebuilds_the_tile_table(B, oracle32):
         assert rel_l2(h.get_state_host()[1], st.g) <= 1e-4
 
 
-def test_bad_rows_are_reported_not_read(B):
+@pytest.mark.parametrize("path", [1, 2], ids=["launches", "persistent"])
+def test_bad_rows_are_reported_not_read(path, B):
     w = inputs.config(0)
-    h = make_gpu(w)
+    h = make_gpu(w, path=path)
     h.init(0)
     m = int(np.min(np.diff(w.row_offsets)))
     with pytest.raises(Exception):
