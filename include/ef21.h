@@ -284,7 +284,8 @@ ef21_status ef21_selftest_exchange_floor(ef21_ctx* ctx, int32_t steps);
 /* Tuning of the persistent path (Algorithm 2 as one kernel; worker i = one thread-block
  * cluster): blocks per cluster (1..8, 0 = automatic), rows per warp batch (4, 8, 16, 32, 0 =
  * automatic) and where the shard rows live (0 registers, 1 shared memory, 2 global memory /
- * L2, -1 = automatic).  A shape that cannot run makes ef21_step fall back (path AUTO) or
+ * L2, -1 = automatic; get_ also reports 3 = global memory through the sampled row numbers of
+ * ef21_step_minibatches).  A shape that cannot run makes ef21_step fall back (path AUTO) or
  * return EF21_ERR_UNSUPPORTED (path PERSISTENT).  get_ reports what the last persistent
  * launch used. */
 ef21_status ef21_set_persistent_shape(ef21_ctx* ctx, int32_t cluster_blocks, int32_t rows_per_batch,

@@ -650,7 +650,7 @@ PersistPlan plan_persistent_body(ef21_ctx* c, bool floor_only, bool roles, int t
             if (src == PK_SRC_REG && ceil_div(rows_cta, rb) > threads / 32) src = PK_SRC_SMEM;
         }
         if (c->pk_src >= 0) src = c->pk_src;
-        if (tau > 0) src = PK_SRC_GMEM;          // sampled rows change every iteration
+        if (tau > 0) src = PK_SRC_SAMPLED;       // sampled rows change every iteration: read through the list
         return rows_cta;
     };
 

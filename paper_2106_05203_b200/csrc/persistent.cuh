@@ -45,7 +45,9 @@ constexpr int PK_MAX_MSGS = 2048;       // n*k words staged in shared memory
 constexpr int PK_SCAN_MAX_MSGS = 128;   // up to this many messages every coordinate thread scans them all
 constexpr int PK_TABLE_MAX_BYTES = 64 * 1024;   // largest [n][ld] message table kept in shared memory
 constexpr unsigned PK_NO_ENTRY = 0xffffffffu;   // table cell without a message (a NaN pattern no finite value has)
-enum { PK_SRC_REG = 0, PK_SRC_SMEM = 1, PK_SRC_GMEM = 2 };
+// where a block's rows come from: registers / shared memory (loaded once), global memory (every iteration), or global
+// memory through a per-iteration list of sampled row numbers (stochastic variant, Algorithm 5)
+enum { PK_SRC_REG = 0, PK_SRC_SMEM = 1, PK_SRC_GMEM = 2, PK_SRC_SAMPLED = 3 };
 
 struct PersistParams {
     const float* A;            // [N][ld], padded, read-only

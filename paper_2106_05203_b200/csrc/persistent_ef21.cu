@@ -5,4 +5,5 @@
 #define PK_PLUS 0
 #define PK_EF 0
 #define PK_FLOOR 0
+#define PK_WITH_SAMPLED 1      // also the instantiations that read sampled rows (Algorithm 5)
 #include "persistent_method.inc"
