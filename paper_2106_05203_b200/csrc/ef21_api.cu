@@ -583,26 +583,26 @@ size_t pk_roles_smem_bytes(int ld, int C, int src, i64 rows_cta, int threads) {
     return b;
 }
 
-PersistPlan plan_persistent_body(ef21_ctx* c, bool floor_only, bool roles, int tau = 0);
+PersistPlan plan_persistent_body(ef21_ctx* c, bool roles, int tau = 0);
 
 // Chooses the kernel body, cluster size, block size, rows per batch and the source of the shard rows; checks
 // that all n clusters can be resident at once (the blocks wait on one another through global memory).
-PersistPlan plan_persistent(ef21_ctx* c, bool floor_only = false) {
+PersistPlan plan_persistent(ef21_ctx* c) {
     // Automatic choice: the serving-warp body for Top-1 (2.8 against 3.0 us per iteration on the mushrooms-shaped
     // workload, 3.7 against 4.6 on the a9a-shaped one, 10.0 against 10.4 on the w8a-shaped one, measured); with more
     // entries per message its k arg-max rounds in one warp cost more than the whole block counting ranks.
     const bool roles_can = c->variant != EF21_VARIANT_EF21_PLUS && c->k <= PK_ROLES_MAX_K;
     const bool roles_first = c->pk_body == 1 || (c->pk_body == 0 && c->k == 1);
     if (roles_can && roles_first) {
-        PersistPlan P = plan_persistent_body(c, floor_only, true);
+        PersistPlan P = plan_persistent_body(c, true);
         if (P.ok || c->pk_body == 1) return P;
     }
     if (c->pk_body == 1) { PersistPlan P; P.ok = false; return P; }
-    return plan_persistent_body(c, floor_only, false);
+    return plan_persistent_body(c, false);
 }
 
 // tau > 0: plan for the stochastic variant (tau sampled rows per worker and iteration, read from global memory).
-PersistPlan plan_persistent_body(ef21_ctx* c, bool floor_only, bool roles, int tau) {
+PersistPlan plan_persistent_body(ef21_ctx* c, bool roles, int tau) {
     PersistPlan P; P.ok = false; P.roles = roles;
     const int ld = (int)c->L.ld;
     if (!c->shards_loaded || ld > 512 || c->k > PK_MAX_K || (i64)c->n * c->k > PK_MAX_MSGS) return P;
@@ -683,12 +683,10 @@ PersistPlan plan_persistent_body(ef21_ctx* c, bool floor_only, bool roles, int t
         if (smem > (size_t)max_smem - 1024) continue;
         PersistKernel kern;
         if (roles)
-            kern = floor_only ? pk_lookup_floor(chunk_slots, rb, src, threads, extra)
-                   : c->variant == EF21_VARIANT_EF ? pk_lookup_ef(chunk_slots, rb, src, threads, extra)
+            kern = c->variant == EF21_VARIANT_EF ? pk_lookup_ef(chunk_slots, rb, src, threads, extra)
                                                    : pk_lookup_ef21(chunk_slots, rb, src, threads, extra);
         else
-            kern = floor_only ? pk_lookup_wide_floor(chunk_slots, rb, src, threads, extra)
-                   : c->variant == EF21_VARIANT_EF ? pk_lookup_wide_ef(chunk_slots, rb, src, threads, extra)
+            kern = c->variant == EF21_VARIANT_EF ? pk_lookup_wide_ef(chunk_slots, rb, src, threads, extra)
                    : (plus ? pk_lookup_plus(chunk_slots, rb, src, threads, extra)
                            : pk_lookup_wide_ef21(chunk_slots, rb, src, threads, extra));
         if (!kern) continue;
@@ -1021,7 +1019,7 @@ ef21_status ef21_step_minibatches(ef21_ctx* c, const int32_t* batches_dev, int32
     if (steps == 0) return EF21_OK;
     if (c->path != EF21_PATH_LAUNCHES && c->k <= PK_ROLES_MAX_K && c->pk_body != 2) {
         if (!c->mb_plan_valid || c->mb_plan_tau != tau) {
-            c->mb_plan = plan_persistent_body(c, false, true, tau);
+            c->mb_plan = plan_persistent_body(c, true, tau);
             c->mb_plan_tau = tau; c->mb_plan_valid = true;
         }
         if (c->mb_plan.ok) {
@@ -1275,8 +1273,16 @@ ef21_status ef21_selftest_exchange_floor(ef21_ctx* c, int32_t steps) {
     if (!c || steps < 1) return EF21_ERR_INVALID_ARG;
     if (!c->shards_loaded || !c->inited) return EF21_ERR_STATE;
     if (c->variant != EF21_VARIANT_EF21) return EF21_ERR_UNSUPPORTED;
-    PersistPlan P = plan_persistent(c, true);
+    // the shape ef21_step itself would launch, with the skeleton kernel of the same instantiation in its place
+    PersistPlan P = plan_persistent(c);
     if (!P.ok) return EF21_ERR_UNSUPPORTED;
+    P.kernel = P.roles ? pk_lookup_floor(P.chunks, P.rb, P.src, P.threads, P.extra)
+                       : pk_lookup_wide_floor(P.chunks, P.rb, P.src, P.threads, P.extra);
+    if (!P.kernel) return EF21_ERR_UNSUPPORTED;
+    int dev = 0, max_smem = 0;
+    CU(cudaGetDevice(&dev));
+    CU(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+    CU(cudaFuncSetAttribute(P.kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem - 1024));
     return run_persistent(c, P, steps);
 }
 
