@@ -450,6 +450,13 @@ def run_ours(args):
         "device_status": r["status"], "f_end": r["f_end"], "persistent_shape": r["shape"],
         "floor_us_per_iteration": time_floor(w, w.k, max(steps, 200)) if r["path"] == 2 else None,
     }
+    if steps != w.T:
+        # the same workload at the iteration count its configuration names (one launch runs them all): what a call costs
+        # per iteration once the launch and the cold start of the kernel are spread over T iterations
+        rT = time_logistic(w, w.k, w.T, warmup)
+        gT = bytes_iter * w.T / (rT["ms"] * 1e-3) / 1e9
+        line["headline_at_T"] = {"steps": w.T, "us_per_iteration": rT["ms"] / w.T * 1e3, "iterations_per_s": whole_job_rate(w.T, world, rT["ms"]),
+                                 "algorithmic_GBps": gT, "frac_of_hbm_peak": gT / peak}
 
     # ---- CPU baseline (rank 0, N = 1 only) ---------------------------------------------------
     if rank == 0 and world == 1 and not args.no_cpu:
