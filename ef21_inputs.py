@@ -219,3 +219,14 @@ def minibatch_rows(seed: int, step: int, row_offsets: np.ndarray, tau: int) -> n
         m = int(row_offsets[i + 1] - row_offsets[i])
         out[i] = rng.choice(m, size=tau, replace=False)
     return out
+
+
+def randk_sets(seed: int, steps: int, n: int, d: int, k: int) -> np.ndarray:
+    """Index sets of the Rand-k compressor: for every step and worker k distinct coordinates drawn uniformly
+    (sampling without replacement), in ascending order, int32 [steps, n, k]."""
+    rng = np.random.default_rng(np.random.PCG64([seed, 104729]))
+    out = np.empty((steps, n, k), dtype=np.int32)
+    for t in range(steps):
+        for i in range(n):
+            out[t, i] = np.sort(rng.choice(d, size=k, replace=False))
+    return out

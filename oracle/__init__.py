@@ -83,6 +83,17 @@ class Oracle:
         self.lib.ef21o_topk(_p(v), _c_int64(d), _c_int64(k), _p(idx), _p(val))
         return idx, val
 
+    def randk(self, v, S, unbiased: bool = False) -> Tuple[np.ndarray, np.ndarray]:
+        """Scaled Rand-k of Example 2 on the index set S (ascending, distinct); unbiased=True: Rand-k itself."""
+        v = self._r(v)
+        S = np.ascontiguousarray(S, dtype=np.int32)
+        k = S.shape[0]
+        idx = np.empty(k, dtype=np.int32)
+        val = np.empty(k, dtype=self.real)
+        fn = self.lib.ef21o_randk_unbiased if unbiased else self.lib.ef21o_randk
+        fn(_p(v), _c_int64(v.shape[0]), _c_int64(k), _p(S), _p(idx), _p(val))
+        return idx, val
+
     # -- objective -----------------------------------------------------------
     def local_loss(self, A, y, x, lam: float) -> float:
         A = self._f32(A); y = self._f32(y); x = self._r(x)
@@ -204,6 +215,16 @@ class State:
         self.o.lib.ef21o_step_minibatch(_c_int32(self.n), _c_int64(self.d), _c_int64(self.k), _p(self.A), _p(self.y),
                                         _p(self.off), _c_double(self.lam), self.o._creal(self.gamma), _p(batch),
                                         _c_int32(batch.shape[1]), *self._args_state())
+
+    def step_randk(self, sets, V=None) -> None:
+        """sets[steps, n, k] (ascending, distinct indices per worker): that many iterations of Algorithm 2 with the
+        scaled Rand-k; V[n, d] (optional) replaces the local gradients."""
+        sets = np.ascontiguousarray(sets, dtype=np.int32)
+        assert sets.ndim == 3 and sets.shape[1] == self.n and sets.shape[2] == self.k
+        Vc = None if V is None else self.o._r(V)
+        self.o.lib.ef21o_step_randk(_c_int32(sets.shape[0]), _c_int32(self.n), _c_int64(self.d), _c_int64(self.k),
+                                    _p(self.A), _p(self.y), _p(self.off), _c_double(self.lam), _p(Vc),
+                                    self.o._creal(self.gamma), _p(sets), *self._args_state())
 
     def round(self, grads) -> None:
         """One message round (no x update) given the local gradients."""

@@ -33,7 +33,9 @@
  * feedback method (Algorithm 4) at the end of the file is pinned by a
  * hand-worked run, the perturbed-iterate identity x - mean e, the contraction
  * of the error, Theorem 3 for the identity compressor and an exact check of
- * every rounding.  The stepsize rule gamma = 1/L is a harness convention:
+ * every rounding.  The diagnostics (||grad f||^2, G^t) are pinned by closed forms at the origin and a planted
+ * distortion; the scaled Rand-k by exact averages over all k-subsets (unbiasedness and second moment of Rand-k,
+ * the contraction of Lemma 8 with equality) and by k = d.  The stepsize rule gamma = 1/L is a harness convention:
  * parity unpinned by the paper.
  */
 #include <math.h>
@@ -292,6 +294,75 @@ void ef21o_step_grads(int32_t steps, int32_t n, int64_t d, int64_t k, const real
         ef21o_x_update(d, gamma, g, x);
         ef21o_round(n, d, k, V, gi, g, idx, val);
     }
+}
+
+/* ------------------------------------------------------------------ */
+/* Scaled Rand-k (Appendix, Lemma 8 and Example 2)                       */
+/* ------------------------------------------------------------------ */
+
+/* Rand-k keeps a uniformly random set S of k coordinates and scales them by d/k, which makes it unbiased
+ * with omega = d/k - 1; Lemma 8 turns an unbiased compressor into a contractive one by the factor
+ * 1/(1 + omega) = k/d.  The two factors cancel: the scaled Rand-k of Example 2 is C(v)_j = v_j for j in S and
+ * 0 elsewhere, in B(k/d).  The set is an input (the caller draws it): S holds k distinct indices in ascending
+ * order.  Output: the k pairs (S_t, v[S_t]). */
+void ef21o_randk(const real* v, int64_t d, int64_t k, const int32_t* S, int32_t* idx, real* val) {
+    (void)d;
+    for (int64_t t = 0; t < k; ++t) { idx[t] = S[t]; val[t] = v[S[t]]; }
+}
+
+/* The unbiased Rand-k itself, C'(v)_j = (d/k) v_j on S (used only to pin the class U(omega) it belongs to). */
+void ef21o_randk_unbiased(const real* v, int64_t d, int64_t k, const int32_t* S, int32_t* idx, real* val) {
+    const real scale = (real)d / (real)k;
+    for (int64_t t = 0; t < k; ++t) { idx[t] = S[t]; val[t] = scale * v[S[t]]; }
+}
+
+/* One message round of Algorithm 2 with the scaled Rand-k in place of Top-k: worker i uses the set
+ * sets[i][0..k).  Node loop and master line as in ef21o_round. */
+void ef21o_randk_round(int32_t n, int64_t d, int64_t k, const real* grads, const int32_t* sets /* [n][k] */,
+                       real* gi, real* g, int32_t* idx, real* val) {
+    real* v = (real*)malloc((size_t)d * sizeof(real));
+    for (int32_t i = 0; i < n; ++i) {
+        const real* gr = grads + (int64_t)i * d;
+        real* gs = gi + (int64_t)i * d;
+        for (int64_t j = 0; j < d; ++j) v[j] = gr[j] - gs[j];
+        int32_t* ix = idx + (int64_t)i * k;
+        real* vl = val + (int64_t)i * k;
+        ef21o_randk(v, d, k, sets + (int64_t)i * k, ix, vl);
+        for (int64_t t = 0; t < k; ++t) gs[ix[t]] = gs[ix[t]] + vl[t];
+    }
+    free(v);
+    /* master: g <- g + (1/n) sum_i c_i, per coordinate in ascending worker order (Algorithm 2, last line) */
+    real* s = (real*)calloc((size_t)d, sizeof(real));
+    unsigned char* touched = (unsigned char*)calloc((size_t)d, 1);
+    for (int32_t i = 0; i < n; ++i)
+        for (int64_t t = 0; t < k; ++t) {
+            int64_t j = idx[(int64_t)i * k + t];
+            s[j] = s[j] + val[(int64_t)i * k + t];
+            touched[j] = 1;
+        }
+    const real inv_n = (real)1 / (real)n;
+    for (int64_t j = 0; j < d; ++j)
+        if (touched[j]) {
+            real p = s[j] * inv_n;
+            g[j] = g[j] + p;
+        }
+    free(s);
+    free(touched);
+}
+
+/* `steps` iterations of Algorithm 2 with the scaled Rand-k; sets[steps][n][k].  V != NULL: the supplied
+ * vectors V[n][d] stand for the local gradients at every step (as in ef21o_step_grads); otherwise the gradients
+ * of Eq. 19 on the shards. */
+void ef21o_step_randk(int32_t steps, int32_t n, int64_t d, int64_t k, const float* A, const float* y,
+                      const int64_t* row_off, double lam, const real* V, real gamma, const int32_t* sets,
+                      real* x, real* gi, real* g, int32_t* idx, real* val) {
+    real* grads = V ? NULL : (real*)malloc((size_t)n * (size_t)d * sizeof(real));
+    for (int32_t t = 0; t < steps; ++t) {
+        ef21o_x_update(d, gamma, g, x);
+        if (!V) ef21o_all_grads(n, d, A, y, row_off, x, lam, grads);
+        ef21o_randk_round(n, d, k, V ? V : grads, sets + (int64_t)t * n * k, gi, g, idx, val);
+    }
+    free(grads);
 }
 
 /* ------------------------------------------------------------------ */

@@ -355,6 +355,66 @@ def test_diagnostics_zero_and_planted_distortion(oracle64):
     assert oracle64.diagnostics(w.A, w.y, w.row_offsets, st.x, w.lam, st.gi)[1] == 0.0
 
 
+# ---------------------------------------------------------------------------
+# Scaled Rand-k (Appendix: Lemma 8, Example 2)
+# ---------------------------------------------------------------------------
+
+def test_randk_exact_moments_over_all_subsets(oracle64):
+    # Rand-k is in U(omega) with omega = d/k - 1: averaged over all C(d, k) equally likely sets, E C'(v) = v and
+    # E||C'(v)||^2 = (d/k)||v||^2 = (1 + omega)||v||^2.  Its scaled version (Lemma 8, factor 1/(1 + omega) = k/d) keeps
+    # the sampled entries as they are, has mean (k/d) v, and meets the bound of Eq. 3 with alpha = k/d with equality:
+    # E||C(v) - v||^2 = (1 - k/d)||v||^2.
+    import itertools
+    rng = np.random.default_rng(2)
+    for d, k in ((5, 2), (6, 3), (7, 1), (4, 4)):
+        v = rng.standard_normal(d)
+        sets = list(itertools.combinations(range(d), k))
+        mean_unb = np.zeros(d); mean_sc = np.zeros(d); sq_unb = 0.0; dist_sc = 0.0
+        for S in sets:
+            iu, vu = oracle64.randk(v, S, unbiased=True)
+            i_s, vs = oracle64.randk(v, S)
+            np.testing.assert_array_equal(iu, S); np.testing.assert_array_equal(i_s, S)
+            cu = np.zeros(d); cu[iu] = vu
+            cs = np.zeros(d); cs[i_s] = vs
+            mean_unb += cu; mean_sc += cs
+            sq_unb += cu @ cu; dist_sc += (cs - v) @ (cs - v)
+            np.testing.assert_array_equal(vs, v[list(S)])             # the two scalings cancel: the entries themselves
+        m = len(sets)
+        np.testing.assert_allclose(mean_unb / m, v, rtol=1e-13)
+        np.testing.assert_allclose(mean_sc / m, (k / d) * v, rtol=1e-13)
+        assert sq_unb / m == pytest.approx((d / k) * (v @ v), rel=1e-13)
+        assert dist_sc / m == pytest.approx((1 - k / d) * (v @ v), rel=1e-13, abs=1e-15)
+
+
+def test_randk_loop_k_equals_d_is_gradient_descent_and_mean_invariant(oracle64):
+    # with S = all coordinates the scaled Rand-k is the identity, so Algorithm 2 is gradient descent (Section 5.2's
+    # remark on k = d); with k < d the master's g stays the mean of the g_i and only the named coordinates move
+    w = inputs.config(0)
+    full = np.tile(np.arange(w.d, dtype=np.int32), (6, w.n, 1))
+    st = oracle_mod.State(oracle64, w.n, w.d, w.d, w.gamma, w.lam, w.A, w.y, w.row_offsets, w.x0)
+    st.init(2)
+    x = np.array(w.x0, dtype=np.float64)
+    g = oracle64.all_grads(w.A, w.y, w.row_offsets, x, w.lam).mean(axis=0)
+    for t in range(6):
+        x = x - w.gamma * g
+        g = oracle64.all_grads(w.A, w.y, w.row_offsets, x, w.lam).mean(axis=0)
+    st.step_randk(full)
+    np.testing.assert_allclose(st.x, x, rtol=1e-12, atol=1e-14)
+    k = 5
+    sets = inputs.randk_sets(3, 12, w.n, w.d, k)
+    st = oracle_mod.State(oracle64, w.n, w.d, k, w.gamma, w.lam, w.A, w.y, w.row_offsets, w.x0)
+    st.init(1)
+    for t in range(12):
+        gi_old = st.gi.copy()
+        st.step_randk(sets[t:t + 1])
+        np.testing.assert_allclose(st.g, st.gi.mean(axis=0), rtol=1e-12, atol=1e-15)
+        grads = st.grads()
+        for i in range(w.n):
+            np.testing.assert_array_equal(st.idx[i], sets[t, i])
+            np.testing.assert_array_equal(np.flatnonzero(st.gi[i] != gi_old[i]), sets[t, i][grads[i][sets[t, i]] != gi_old[i][sets[t, i]]])
+            np.testing.assert_allclose(st.gi[i][sets[t, i]], grads[i][sets[t, i]], rtol=1e-15)      # g_i takes the gradient's entries
+
+
 def test_theory_constants_closed_forms():
     # Section 3.3 and Example 1: sqrt(beta/theta) = sqrt(1-alpha)/(1-sqrt(1-alpha)) = (1+sqrt(1-alpha))/alpha - 1.
     for alpha in (1 / 300, 4 / 64, 0.5, 0.999):
