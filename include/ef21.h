@@ -155,6 +155,16 @@ ef21_status ef21_step_grads(ef21_ctx* ctx, const float* V_dev, int32_t steps);
 ef21_status ef21_step_minibatches(ef21_ctx* ctx, const int32_t* batches_dev, int32_t tau, int32_t steps);
 ef21_status ef21_step_minibatch(ef21_ctx* ctx, const int32_t* batch_dev, int32_t tau);
 
+/* `steps` iterations of Algorithm 2 with the scaled Rand-k compressor in place of Top-k (Appendix, Lemma 8 and
+ * Example 2: Rand-k, which keeps k uniformly drawn coordinates times d/k, scaled by 1/(1 + omega) = k/d -- the
+ * factors cancel, the compressor keeps the drawn entries as they are and lies in B(k/d)).  The library draws
+ * nothing: sets_dev[steps][n][k] holds, for every iteration and worker, the k drawn coordinates, distinct and in
+ * ascending order (int32); an entry outside [0, d) or out of order is replaced and EF21_ERR_INVALID_ARG is
+ * recorded in the status word.  V_dev[n][d], if not NULL, stands for the local gradients at every iteration (as in
+ * ef21_step_grads); otherwise the gradients of the objective on the loaded shards are used.  Launch path;
+ * EF21_VARIANT_EF21 only.  Given the same gradients the result is bit-identical to the plain definition. */
+ef21_status ef21_step_randk(ef21_ctx* ctx, const float* V_dev, const int32_t* sets_dev, int32_t steps);
+
 /* grad f_i(x) for the current x and all workers, written to grads_out_dev[n][d]
  * (Eq. 19 differentiated; state is not changed). */
 ef21_status ef21_local_grads(ef21_ctx* ctx, float* grads_out_dev);

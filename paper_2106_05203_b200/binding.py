@@ -42,6 +42,7 @@ SIGNATURES = {
     "ef21_step_grads": (ctypes.c_int, [_vp, _vp, _i32]),
     "ef21_step_minibatch": (ctypes.c_int, [_vp, _vp, _i32]),
     "ef21_step_minibatches": (ctypes.c_int, [_vp, _vp, _i32, _i32]),
+    "ef21_step_randk": (ctypes.c_int, [_vp, _vp, _vp, _i32]),
     "ef21_local_grads": (ctypes.c_int, [_vp, _vp]),
     "ef21_topk_workspace_bytes": (_sz, [_i32, _i64, _i32]),
     "ef21_topk": (ctypes.c_int, [_vp, _i32, _i64, _i32, _vp, _vp, _vp, _sz, _vp]),
@@ -213,6 +214,17 @@ class EF21:
         _check(_lib.ef21_step_minibatches(self._h, _ptr(batches), int(batches.shape[2]), int(batches.shape[0])),
                "ef21_step_minibatches")
         self._keep_batch = batches
+
+    def step_randk(self, sets: torch.Tensor, V: Optional[torch.Tensor] = None) -> None:
+        """sets[steps, n, k] int32 (ascending, distinct coordinates per worker): that many iterations with the scaled
+        Rand-k compressor; V[n, d] (optional) replaces the local gradients."""
+        if not (sets.is_cuda and sets.dtype == torch.int32 and sets.is_contiguous() and sets.dim() == 3
+                and sets.shape[1] == self.n and sets.shape[2] == self.k):
+            raise TypeError("sets must be a contiguous int32 CUDA tensor of shape [steps, n, k]")
+        if V is not None:
+            _dev_f32(V, (self.n, self.d))
+        _check(_lib.ef21_step_randk(self._h, _ptr(V), _ptr(sets), int(sets.shape[0])), "ef21_step_randk")
+        self._keep_batch = (sets, V)
 
     def local_grads(self) -> torch.Tensor:
         out = torch.empty((self.n, self.d), dtype=torch.float32, device=self.device)

@@ -22,6 +22,27 @@ __global__ void apply_messages_kernel(const int* __restrict__ idx, const float* 
     *p = __fadd_rn(*p, val[e]);
 }
 
+// Scaled Rand-k (Appendix, Lemma 8 and Example 2: Rand-k times 1/(1 + omega) keeps the k sampled entries as they
+// are): message entry t of worker i is (S, a[S] - g_i[S]) with S = sets[i][t], and g_i[S] takes the sum.  The sets are
+// an input: k distinct indices in ascending order per worker.  An index outside [0, d), or one that does not exceed
+// its predecessor, is reported through the status word and replaced by position t (never dereferenced as given).
+__global__ void randk_select_kernel(const float* __restrict__ a, i64 pitch_a, float* __restrict__ gi, i64 ld,
+                                    const int* __restrict__ sets, i64 total, int k, i64 d,
+                                    int* __restrict__ idx_out, float* __restrict__ val_out, unsigned* status) {
+    const i64 e = blockIdx.x * (i64)blockDim.x + threadIdx.x;
+    if (e >= total) return;
+    const i64 i = e / k;
+    const int t = (int)(e - i * k);
+    int j = sets[e];
+    const bool bad = j < 0 || (i64)j >= d || (t > 0 && sets[e - 1] >= j);
+    if (bad) { record_error(status, 1u /* EF21_ERR_INVALID_ARG */); j = t; }
+    float* p = gi + i * ld + j;
+    const float v = __fsub_rn(a[i * pitch_a + j], *p);
+    idx_out[e] = j; val_out[e] = v;
+    flag_nonfinite(status, v);
+    *p = __fadd_rn(*p, v);
+}
+
 // off[i][b] = first position in worker i's ascending index list with idx >= b * AGG_TILE,
 // for b = 0 .. ntiles (so tile b owns entries [off[i][b], off[i][b+1])).
 __global__ void agg_offsets_kernel(const int* __restrict__ idx, int n, int k, int ntiles,

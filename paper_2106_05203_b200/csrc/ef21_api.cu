@@ -1042,6 +1042,27 @@ ef21_status ef21_step_minibatch(ef21_ctx* c, const int32_t* batch_dev, int32_t t
     return ef21_step_minibatches(c, batch_dev, tau, 1);
 }
 
+ef21_status ef21_step_randk(ef21_ctx* c, const float* V_dev, const int32_t* sets_dev, int32_t steps) {
+    if (!c || !sets_dev || steps < 0) return EF21_ERR_INVALID_ARG;
+    if (!c->inited || (!V_dev && !c->shards_loaded)) return EF21_ERR_STATE;
+    if (c->variant != EF21_VARIANT_EF21) return EF21_ERR_UNSUPPORTED;
+    const i64 total = (i64)c->n * c->k;
+    for (int t = 0; t < steps; ++t) {
+        EF(enqueue_x_update(c));
+        if (!V_dev) EF(enqueue_grads(c, false));
+        const float* a = V_dev ? V_dev : c->at<float>(c->L.grad);
+        const i64 pitch = V_dev ? c->d : c->L.ld;
+        randk_select_kernel<<<(unsigned)ceil_div(total, 256), 256, 0, c->stream>>>(
+            a, pitch, c->gi(), c->L.ld, sets_dev + (size_t)t * total, total, c->k, c->d, c->msg_idx(), c->msg_val(), c->status());
+        c->launches += 1;
+        CU(cudaGetLastError());
+        c->agg_off_ready = false;
+        EF(enqueue_round_aggregate(c, false));
+    }
+    c->last_path = EF21_PATH_LAUNCHES;
+    return EF21_OK;
+}
+
 ef21_status ef21_local_grads(ef21_ctx* c, float* grads_out_dev) {
     if (!c || !grads_out_dev) return EF21_ERR_INVALID_ARG;
     if (!c->shards_loaded) return EF21_ERR_STATE;
