@@ -33,6 +33,7 @@
 // block skips work but keeps arriving at the cluster barriers, so the kernel always terminates.
 #pragma once
 #include <cooperative_groups.h>
+#include <cuda/std/type_traits>
 
 #include "common.cuh"
 
