@@ -22,11 +22,13 @@
 //      coordinate thread adds the matching values in ascending worker order (few messages), or warp 0
 //      folds the messages worker by worker into running sums (many messages): g += (1/n) sum c_i
 //
-// The kernel itself is persistent_body.inc; it is compiled three times (persistent_ef21.cu,
-// persistent_plus.cu, persistent_ef.cu): Algorithm 2 as described above, EF21+ (Algorithm 3: a second
-// selection on grad_i, the two distortions, per-block replicas of all g_i and a dense mean) and the
-// original EF (Algorithm 4: the leader compresses e_i + gamma grad_i, the messages move x directly).
-// This header holds what the three share.
+// Two bodies implement these steps.  persistent_body.inc takes every step with the whole block between block
+// barriers, as listed above; persistent_roles.inc lets the last warp of a block serve it (steps 1, 3, 4, 5 in one
+// warp, four coordinates per lane) while the other warps only sweep rows (step 2) between two named barriers.
+// Each body is compiled once per method, one translation unit each (persistent_*.cu): Algorithm 2 as described
+// above, EF21+ (Algorithm 3: a second selection on grad_i, the two distortions, per-block replicas of all g_i and a
+// dense mean; whole-block body only), the original EF (Algorithm 4: the leader compresses e_i + gamma grad_i, the
+// messages move x directly) and the exchange skeleton (a measuring aid).  This header holds what they share.
 //
 // All summation orders are fixed by the launch shape, so two runs give identical bits.  A wait
 // that exceeds its spin limit records EF21_ERR_TIMEOUT in the status word; from then on every
