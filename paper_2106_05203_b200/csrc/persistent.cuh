@@ -144,6 +144,41 @@ __device__ __forceinline__ float comp_of(const float4& v, int c) {
 // its own value; 0 marks a word that no iteration has written (the array is cleared once, at creation).
 __device__ __forceinline__ unsigned next_epoch(unsigned e) { return e >= 65535u ? 1u : e + 1u; }
 
+// Top-k of up to 128 entries held four per lane (lane L owns entries 4L .. 4L+3 in v4), by one warp, for vectors of at
+// most 128 coordinates.  Every lane first orders its own four entries by (|.| bits descending, index ascending); a round
+// then is the warp maximum of the lanes' best remaining keys, the warp minimum of the indices that hold it (the lower
+// index wins a tie), and the owner dropping that entry -- two redux and a handful of predicated moves, nothing is
+// recomputed.  pad_bits: bit e set = entry 4L+e lies beyond d and is never taken.  Returns the lane's 4-bit mask of
+// selected entries; position receives the number of selected entries in lower lanes, so that a lane can emit its picks
+// in ascending index order at position, position + 1, ...
+__device__ __forceinline__ unsigned warp_topk_four_per_lane(const float4& v4, unsigned pad_bits, int k, int lane, int& position) {
+    // composite (key, 3 - e): larger is better; -1 marks an entry that cannot be taken
+    long long c[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const long long key = ((pad_bits >> e) & 1u) ? -1ll : (long long)mag_key(comp_of(v4, e));
+        c[e] = key < 0 ? -1ll : ((key << 2) | (long long)(3 - e));
+    }
+    auto order = [&](int a, int b) { const long long hi = max(c[a], c[b]), lo = min(c[a], c[b]); c[a] = hi; c[b] = lo; };
+    order(0, 1); order(2, 3); order(0, 2); order(1, 3); order(1, 2);
+    int k0 = (int)(c[0] >> 2), k1 = (int)(c[1] >> 2), k2 = (int)(c[2] >> 2), k3 = (int)(c[3] >> 2);       // -1 stays -1
+    int e0 = 3 - (int)(c[0] & 3), e1 = 3 - (int)(c[1] & 3), e2 = 3 - (int)(c[2] & 3), e3 = 3 - (int)(c[3] & 3);
+    unsigned mask = 0u;
+    for (int round = 0; round < k; ++round) {
+        const int wk = __reduce_max_sync(0xffffffffu, k0);
+        const unsigned mine = (k0 == wk && k0 >= 0) ? (unsigned)(4 * lane + e0) : 0xffffffffu;
+        const unsigned widx = __reduce_min_sync(0xffffffffu, mine);
+        if (mine == widx && mine != 0xffffffffu) {
+            mask |= 1u << e0;
+            k0 = k1; e0 = e1; k1 = k2; e1 = e2; k2 = k3; e2 = e3; k3 = -1;
+        }
+    }
+    const unsigned cnt = (unsigned)__popc(mask), lt = (1u << lane) - 1u;
+    const unsigned b0 = __ballot_sync(0xffffffffu, cnt & 1u), b1 = __ballot_sync(0xffffffffu, cnt & 2u), b2 = __ballot_sync(0xffffffffu, cnt & 4u);
+    position = __popc(b0 & lt) + 2 * __popc(b1 & lt) + 4 * __popc(b2 & lt);
+    return mask;
+}
+
 typedef void (*PersistKernel)(const PersistParams);
 
 // One lookup per method (each in a translation unit of its own, so that they compile side by side):
