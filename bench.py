@@ -38,10 +38,10 @@ FALLBACK_HBM_GBS = 6650.0
 # registers, shared memory or L2), so the per-launch figure holds for any step count.  None: not captured for the
 # kernel as it stands.
 NCU_TRAFFIC = {
-    # persistent_kernel<1,16,REG,256,0>, launches of 2,000 iterations: 3,735,552 B read (both launches), 0 B written
-    "headline": {"per": "launch", "bytes": 3735552},
-    # persistent_kernel<3,4,GMEM,512,0>, launches of 50 iterations: 30,100,359,424 B read + 3,445,760 B written
-    "hbm_persistent": {"per": "iteration", "bytes": 602076104},
+    # persistent_kernel<1,16,REG,256,0>, launches of 2,000 iterations: 3,744,256 B read, 0 B written
+    "headline": {"per": "launch", "bytes": 3744256},
+    # persistent_kernel<3,4,GMEM,512,0>, launches of 50 iterations: 30,100,754,176 B read + 3,494,400 B written
+    "hbm_persistent": {"per": "iteration", "bytes": 602084972},
     # st_collect_kernel<true> captured at n = 16 workers (537.12 MB read + 4.64 MB written per launch), scaled by
     # 64 / 16: the pass reads every vector once, so its traffic grows with the number of workers
     "stress_collect": {"per": "iteration", "bytes": 2167040000},
