@@ -463,6 +463,41 @@ def test_persistent_body_choice(B):
     assert e.value.status == 7
 
 
+@pytest.mark.parametrize("body", [1, 2], ids=["serving-warp", "whole-block"])
+def test_persistent_epochs_wrap_around(body, B, oracle32):
+    # the 16-bit epoch of the message words runs on from launch to launch and wraps from 65,535 to 1: a run that
+    # crosses the wrap inside a launch, and one that crosses it between launches, give the same bits
+    w = inputs.config(0, k=2)
+    outs = []
+    for chunks in ((65500, 200), (65535, 1, 164), (30000, 35700)):
+        h = make_gpu(w, k=2, path=2); h.set_persistent_body(body); h.init(0)
+        for s_ in chunks:
+            h.step(s_)
+        assert h.poll() == 0
+        outs.append(h.get_state_host())
+    for other in outs[1:]:
+        for a_, b_ in zip(outs[0], other):
+            np.testing.assert_array_equal(a_, b_)
+    assert np.all(np.isfinite(outs[0][0]))
+    # long after convergence the iterate is a stationary point of the oracle's objective as well
+    grads = oracle32.all_grads(w.A, w.y, w.row_offsets, outs[0][0], w.lam).astype(np.float64)
+    assert np.linalg.norm(grads.mean(axis=0)) <= 1e-4
+
+
+def test_two_handles_share_the_kernels(B, oracle32):
+    # two handles of different shapes take turns on one stream: each keeps its own cached launch plan, message slots
+    # and epochs, and both follow the oracle
+    wa, wb = inputs.config(0, k=1), inputs.config(1)
+    ha, hb = make_gpu(wa, k=1, path=2), make_gpu(wb, path=2)
+    sa, sb = make_oracle_state(oracle32, wa, k=1), make_oracle_state(oracle32, wb)
+    ha.init(0); hb.init(0); sa.init(0); sb.init(0)
+    for _ in range(4):
+        ha.step(7); hb.step(5); sa.step(7); sb.step(5)
+    assert rel_l2(ha.get_state_host()[0], sa.x) <= 1e-4
+    assert rel_l2(hb.get_state_host()[0], sb.x) <= 1e-4
+    assert ha.poll() == 0 and hb.poll() == 0
+
+
 def test_persistent_many_steps_in_one_launch_equals_single_steps(B):
     w = inputs.config(1)
     a = make_gpu(w, path=2); a.init(0); a.step(300)
