@@ -131,3 +131,55 @@ def test_persistent_ef21_plus_many_steps_in_one_launch_equal_single_steps(B):
         outs.append(h.get_state_host() + (h.get_plus_choice(),))
     for a_, b_ in zip(outs[0], outs[1]):
         np.testing.assert_array_equal(a_, b_)
+
+
+@pytest.mark.parametrize("n,d,k", [(6, 64, 3), (20, 112, 1), (40, 100, 2)], ids=["n6", "n20", "n40"])
+def test_persistent_ef21_plus_takes_the_plain_branch(n, d, k, B, oracle32):
+    """Workers whose g_i is far from their gradient must fall back to the plain compressor (B_i < M_i, Algorithm 3):
+    their row of the replicas restarts from zero.  Every other worker is put there by hand, the rest keep their state,
+    so one launch sees both branches side by side (n = 40: more workers than one ballot covers)."""
+    w = inputs.make_logistic("plusbranch", n=n, d=d, N=n * 30, k=k, seed=4000 + n, features="gauss", flip=0.1, gamma=0.05, T=10)
+    h = make_gpu(w, k=k, path=2); h.set_variant(B.VARIANT_EF21_PLUS)
+    st = make_oracle_state(oracle32, w, k=k)
+    h.init(0); st.init(0)
+    rng = np.random.default_rng(n)
+    seen = set()
+    for t in range(6):
+        if t % 2 == 0:
+            st.gi[t // 2 % 2::2] = (25.0 * rng.standard_normal(st.gi[t // 2 % 2::2].shape)).astype(np.float32)
+        set_gpu_state_from_oracle(h, st)
+        gi_old = st.gi.copy()
+        h.step(1); st.plus_step(1)
+        assert h.last_path == B.PATH_PERSISTENT
+        x, g, gi, li, lv = h.get_state_host()
+        choice = h.get_plus_choice()
+        for i in np.flatnonzero(choice != st.choice):
+            # only two distortions within the effect of the gradient tolerance of each other may be ordered differently
+            gd = st.grads()[i].astype(np.float64)
+            vm = gd - gi_old[i]
+            im, _ = oracle32.topk(vm.astype(np.float32), k)
+            ib, _ = oracle32.topk(gd.astype(np.float32), k)
+            rest_m = vm.copy(); rest_m[im] = 0.0
+            rest_b = gd.copy(); rest_b[ib] = 0.0
+            M, Bd = float(rest_m @ rest_m), float(rest_b @ rest_b)
+            assert abs(M - Bd) <= 1e-4 * max(M, Bd), (t, i, M, Bd)
+        if not np.array_equal(choice, st.choice):
+            continue
+        if t % 2 == 0:
+            assert np.all(st.choice[t // 2 % 2::2] == 1), "a g_i of norm 25 sqrt(d) must lose against the plain compressor"
+        seen |= set(st.choice.tolist())
+        grads = st.grads()
+        for i in range(n):
+            tol = 1e-5 * np.max(np.abs(grads[i]))
+            if st.choice[i] == 1:
+                # C(grad_i): index set up to near-ties, values within the gradient tolerance, all other entries exactly 0
+                assert np.count_nonzero(gi[i]) <= k
+                if np.array_equal(li[i], st.idx[i]):
+                    assert np.max(np.abs(lv[i] - st.val[i])) <= tol
+                    assert np.max(np.abs(gi[i] - st.gi[i])) <= tol
+            elif np.array_equal(li[i], st.idx[i]):
+                assert np.max(np.abs(gi[i] - st.gi[i])) <= tol + 4e-6 * np.max(np.abs(gi_old[i]))
+        assert np.max(np.abs(g - st.g)) <= 1e-5 * max(np.max(np.abs(st.gi)), 1e-30)
+        assert rel_l2(x, st.x) <= 1e-5
+    assert seen == {0, 1}
+    assert h.poll() == 0
