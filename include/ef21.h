@@ -133,7 +133,12 @@ ef21_status ef21_init_grads(ef21_ctx* ctx, const float* V_dev, int32_t mode);
  * replayed as a CUDA graph that the handle captures once (on a stream of its own; the CUDA runtime
  * keeps the graph's resources until ef21_destroy) and launches into the handle's stream; if that
  * stream is itself being captured, or the capture fails, the kernels are launched one by one.
- * Results are identical either way. */
+ * Results are identical either way.
+ * On the persistent path one launch holds all of its thread-block clusters on the device at once.  Launches
+ * of several handles are therefore kept from overlapping: a persistent launch on another stream than the
+ * device's previous one is ordered (on the device, by an event; the host does not wait) after everything
+ * that stream holds so far.  The device meant is the one current at ef21_create; keep it current for the
+ * handle's calls. */
 ef21_status ef21_step(ef21_ctx* ctx, int32_t steps);
 /* The same loop with grad f_i replaced by the caller's V_dev[n][d], re-used unchanged at
  * each of the `steps` iterations (the static input sequence of Section 3.1); call with

@@ -170,6 +170,7 @@ struct PersistPlan {
 struct ef21_ctx {
     int n; i64 d; int k; float gamma, lambda; i64 N;
     cudaStream_t stream;
+    int device;         // the device that was current at ef21_create
     char* ws;
     Layout L;
     bool shards_loaded, inited;
@@ -712,7 +713,50 @@ PersistPlan plan_persistent_body(ef21_ctx* c, bool roles, int tau) {
     return P;
 }
 
+// Persistent launches of different handles must not overlap on a device.  Each needs all of its clusters resident at
+// once (they wait on one another through global memory); two launches that each got part of the SMs would wait for
+// the other's until their bounded waits expire.  Launches on one stream are ordered by the stream.  A launch on another
+// stream than the device's last persistent launch first waits (on the device, not on the host) for everything enqueued
+// on that stream so far.
+struct PersistGate {
+    std::mutex mu;
+    bool any = false;              // a persistent launch has been enqueued on this device
+    bool detached = false;         // its handle is gone: `ev` stands for the work, the stream is not touched again
+    cudaStream_t last_stream = nullptr;
+    cudaEvent_t ev = nullptr;
+};
+constexpr int GATE_DEVICES = 64;
+PersistGate g_gate[GATE_DEVICES];
+
+PersistGate* gate_of_device(int dev) { return (dev >= 0 && dev < GATE_DEVICES) ? &g_gate[dev] : nullptr; }
+
+ef21_status gate_order_after_last(PersistGate* G, cudaStream_t stream) {
+    if (!G->any || (!G->detached && G->last_stream == stream)) return EF21_OK;
+    if (!G->ev) CU(cudaEventCreateWithFlags(&G->ev, cudaEventDisableTiming));
+    if (!G->detached) CU(cudaEventRecord(G->ev, G->last_stream));
+    CU(cudaStreamWaitEvent(stream, G->ev, 0));
+    return EF21_OK;
+}
+
+// Called when a handle goes away: its stream may be destroyed by the caller afterwards, so what it has enqueued is
+// pinned to the event now.
+void gate_forget_stream(int dev, cudaStream_t stream) {
+    PersistGate* G = gate_of_device(dev);
+    if (!G) return;
+    std::lock_guard<std::mutex> lock(G->mu);
+    if (!G->any || G->detached || G->last_stream != stream) return;
+    if (!G->ev && cudaEventCreateWithFlags(&G->ev, cudaEventDisableTiming) != cudaSuccess) { cudaGetLastError(); G->any = false; return; }
+    if (cudaEventRecord(G->ev, stream) != cudaSuccess) { cudaGetLastError(); G->any = false; return; }
+    G->detached = true;
+}
+
 ef21_status run_persistent(ef21_ctx* c, const PersistPlan& P, int steps, const int* batch = nullptr, int tau = 0) {
+    PersistGate* G = gate_of_device(c->device);
+    std::unique_lock<std::mutex> gate_lock;
+    if (G) {
+        gate_lock = std::unique_lock<std::mutex>(G->mu);
+        EF(gate_order_after_last(G, c->stream));
+    }
     PersistParams p;
     p.batch = batch; p.tau = tau;
     p.A = c->at<float>(c->L.A); p.y = c->at<float>(c->L.y); p.row_off = c->at<i64>(c->L.row_off);
@@ -736,6 +780,7 @@ ef21_status run_persistent(ef21_ctx* c, const PersistPlan& P, int steps, const i
     cfg.attrs = attr; cfg.numAttrs = 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, P.kernel, p);
     if (e != cudaSuccess) { cudaGetLastError(); return EF21_ERR_CUDA; }
+    if (G) { G->any = true; G->detached = false; G->last_stream = c->stream; }
     c->launches += 1;
     c->pk_epoch = (unsigned)(((i64)c->pk_epoch + steps - 1) % 65535) + 1u;
     c->pk_par = (c->pk_par + (unsigned)steps) & 1u;
@@ -782,6 +827,8 @@ ef21_status ef21_create(ef21_ctx** out, int32_t n, int64_t d, int32_t k, float g
     if (!c) return EF21_ERR_INVALID_ARG;
     c->n = n; c->d = d; c->k = k; c->gamma = gamma; c->lambda = lambda; c->N = total_rows;
     c->stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    c->device = -1;
+    if (cudaGetDevice(&c->device) != cudaSuccess) { cudaGetLastError(); c->device = -1; }
     c->ws = static_cast<char*>(workspace_dev);
     c->L = L;
     c->shards_loaded = false; c->inited = false; c->num_tiles = 0;
@@ -811,6 +858,7 @@ ef21_status ef21_create(ef21_ctx** out, int32_t n, int64_t d, int32_t k, float g
 
 void ef21_destroy(ef21_ctx* ctx) {
     if (!ctx) return;
+    gate_forget_stream(ctx->device, ctx->stream);
     if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
     if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
     if (ctx->aux_stream) cudaStreamDestroy(ctx->aux_stream);

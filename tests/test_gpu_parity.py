@@ -498,6 +498,34 @@ def test_two_handles_share_the_kernels(B, oracle32):
     assert ha.poll() == 0 and hb.poll() == 0
 
 
+def test_two_handles_on_two_streams_are_kept_apart(B):
+    # 120 blocks each on 148 SMs: the two launches cannot be resident together, and each needs all of its clusters at
+    # once.  The library orders a persistent launch after the device's previous one when the streams differ, so both
+    # run to the end and give the bits of a run alone.
+    w = inputs.config(2, k=1)
+    alone = make_gpu(w, k=1, path=2); alone.init(0); alone.step(400)
+    want = alone.get_state_host()
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    hs = []
+    A_t, y_t, x_t = dev(w.A), dev(w.y), dev(w.x0)          # alive until the end of the test: the handles read them on their streams
+    torch.cuda.synchronize()
+    for s in (s1, s2):
+        h = B.EF21(w.n, w.d, 1, w.gamma, w.lam, total_rows=w.N, stream=s)
+        h.set_path(2)
+        h.load_shards(A_t, y_t, w.row_offsets); h.set_x(x_t); h.init(0)
+        hs.append(h)
+    torch.cuda.synchronize()
+    for _ in range(4):                     # no host synchronisation between the calls: the launches queue up
+        hs[0].step(100); hs[1].step(100)
+    for h in hs:
+        assert h.poll() == 0 and h.last_path == B.PATH_PERSISTENT
+        for u, v in zip(h.get_state_host(), want):
+            np.testing.assert_array_equal(u, v)
+    hs[1].close()                          # the last launch was this handle's: its stream must not be touched again
+    hs[0].step(5)
+    assert hs[0].poll() == 0
+
+
 def test_persistent_many_steps_in_one_launch_equals_single_steps(B):
     w = inputs.config(1)
     a = make_gpu(w, path=2); a.init(0); a.step(300)
