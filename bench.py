@@ -38,10 +38,10 @@ FALLBACK_HBM_GBS = 6650.0
 # registers, shared memory or L2), so the per-launch figure holds for any step count.  None: not captured for the
 # kernel as it stands.
 NCU_TRAFFIC = {
-    # persistent_kernel<1,16,REG,256,0>, launches of 2,000 iterations: 3,744,256 B read, 0 B written
-    "headline": {"per": "launch", "bytes": 3744256},
-    # persistent_kernel<3,4,GMEM,512,0>, launches of 50 iterations: 30,103,342,592 B read + 4,387,840 B written
-    "hbm_persistent": {"per": "iteration", "bytes": 602154609},
+    # persistent_kernel<1,16,REG,256,0>, launches of 2,000 iterations: 3,746,048 B read, 0 B written
+    "headline": {"per": "launch", "bytes": 3746048},
+    # persistent_kernel<3,4,GMEM,512,0>, launches of 50 iterations: 30,100,547,840 B read + 4,156,416 B written
+    "hbm_persistent": {"per": "iteration", "bytes": 602094085},
     # st_collect_kernel<true> captured at n = 16 workers (537.12 MB read + 4.64 MB written per launch), scaled by
     # 64 / 16: the pass reads every vector once, so its traffic grows with the number of workers
     "stress_collect": {"per": "iteration", "bytes": 2167040000},

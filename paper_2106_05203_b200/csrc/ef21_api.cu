@@ -589,8 +589,8 @@ PersistPlan plan_persistent_body(ef21_ctx* c, bool roles, int tau = 0);
 // Chooses the kernel body, cluster size, block size, rows per batch and the source of the shard rows; checks
 // that all n clusters can be resident at once (the blocks wait on one another through global memory).
 PersistPlan plan_persistent(ef21_ctx* c) {
-    // Automatic choice: the serving-warp body for Top-1 (2.8 against 3.0 us per iteration on the mushrooms-shaped
-    // workload, 3.7 against 4.6 on the a9a-shaped one, 10.0 against 10.4 on the w8a-shaped one, measured); with more
+    // Automatic choice: the serving-warp body for Top-1 (2.6 against 3.2 us per iteration on the mushrooms-shaped
+    // workload, 3.4 against 4.0 on the a9a-shaped one, the same 10.4 on the w8a-shaped one, measured); with more
     // entries per message its k arg-max rounds in one warp cost more than the whole block counting ranks.
     const bool roles_can = c->variant != EF21_VARIANT_EF21_PLUS && c->k <= PK_ROLES_MAX_K;
     const bool roles_first = c->pk_body == 1 || (c->pk_body == 0 && c->k == 1);
