@@ -211,7 +211,9 @@ def run_reference(args):
     line = {
         "impl": "reference", "metric": METRIC, "value": its, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
         "warmup": warmup, "ms_per_step": dt / steps * 1e3, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f64 gradients, f32 state", "data": "synthetic",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "dtype_note": "state, differences, Top-k, aggregation and x update in fp32 as in the GPU arm; the oracle forms every "
+                      "loss and gradient sum in fp64 and rounds it once to fp32",
         "config": {"workload": workload_string(w)},
         "cpu_baseline": {"value": its, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": its, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
