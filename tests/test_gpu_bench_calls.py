@@ -9,7 +9,8 @@
     messages and g_i of sampled workers bit for bit against 50 oracle steps;
   * several steps in one call on long Student-t vectors (the second-stream path with the threshold estimated ahead),
     bit for bit;
-  * shards larger than L2 (600 MB), iteration by iteration.
+  * shards larger than L2 (600 MB), iteration by iteration;
+  * the lines for Algorithms 3 and 4 (EF21+ and EF on the mushrooms-shaped workload, 500 iterations, persistent kernels).
 """
 import numpy as np
 import pytest
@@ -170,4 +171,51 @@ def test_lockstep_shards_beyond_l2(path, B, oracle32):
     want = st.grads()
     for i in range(w.n):
         assert rel_l2(got[i], want[i]) <= 1e-5
+    assert h.poll() == 0
+
+
+@pytest.mark.parametrize("variant", ["ef21_plus", "ef"])
+def test_variant_calls_of_the_benchmark(variant, B, oracle32, oracle64):
+    """The benchmark's lines for Algorithms 3 and 4 on the mushrooms-shaped workload, automatic path (the persistent kernel
+    of the variant), from the variant's own start: 500 iterations, free-running, 50 per call.
+
+    After every call x must be within 1e-4 of the oracle's.  Top-k makes the trajectory discontinuous: the oracle with
+    its state in fp64 parts from the oracle with its state in fp32 by 6e-4 around iteration 250 of the EF21+ run and comes
+    back to 1e-4 by iteration 500 (rounding differences of 1e-7 in the state decide a near-tie some iterations later).
+    Where the two oracles, running freely from one state, have parted by more than 1e-5, fp32 arithmetic cannot decide
+    the trajectory; there, and only there, the GPU may part too (by no more than ten times as much), and all three
+    continue from the fp32 oracle's state."""
+    w = inputs.config(1)
+    h = make_gpu(w)
+    if variant == "ef21_plus":
+        h.set_variant(B.VARIANT_EF21_PLUS)
+        st, wide = make_oracle_state(oracle32, w), make_oracle_state(oracle64, w)
+        h.init(0); st.init(0); wide.init(0)
+        fields = ("x", "g", "gi")
+        advance = lambda s_, n_: s_.plus_step(n_)
+        rebase = lambda: set_gpu_state_from_oracle(h, st)
+    else:
+        h.set_variant(B.VARIANT_EF)
+        st = oracle_mod.EFState(oracle32, w.n, w.d, w.k, w.gamma, w.lam, w.A, w.y, w.row_offsets, w.x0)
+        wide = oracle_mod.EFState(oracle64, w.n, w.d, w.k, w.gamma, w.lam, w.A, w.y, w.row_offsets, w.x0)
+        h.init(B.INIT_ZERO); st.init(); wide.init()
+        fields = ("x", "e")
+        advance = lambda s_, n_: s_.step(n_)
+        rebase = lambda: h.set_state(dev(st.x), None, dev(st.e))
+    undecidable = []
+    for done in range(0, 500, 50):
+        h.step(50); advance(st, 50); advance(wide, 50)
+        assert h.last_path == B.PATH_PERSISTENT
+        parted = rel_l2(h.get_state_host()[0], st.x)
+        if parted > 1e-4:
+            between_oracles = rel_l2(wide.x, st.x)
+            assert between_oracles > 1e-5 and parted <= 10 * between_oracles, (done, parted, between_oracles)
+            undecidable.append(done)
+            rebase()
+            for f in fields:                      # all three continue from one state
+                getattr(wide, f)[...] = getattr(st, f)
+    print(f"{variant}: stretches the arithmetic cannot decide: {undecidable}")
+    assert len(undecidable) <= 3
+    assert rel_l2(h.get_state_host()[0], st.x) <= 1e-4
+    assert h.eval()[0] == pytest.approx(st.loss(), rel=1e-4)
     assert h.poll() == 0
