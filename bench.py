@@ -496,6 +496,29 @@ def run_ours(args):
         re_ = time_logistic(wp, wp.k, 500, 10, variant=B.VARIANT_EF)
         others.append({"workload": f"EF (Algorithm 4) on configs[{HEADLINE}] {wp.name} Top-{wp.k}", "iterations_per_s": 500 / (re_["ms"] * 1e-3),
                        "us_per_iteration": re_["ms"] / 500 * 1e3, "launches": re_["launches"], "f_end": re_["f_end"]})
+        # stochastic EF21 (Algorithm 5): tau sampled rows per worker and iteration, 500 iterations in one call
+        for tau in (32, 128):
+            hm = B.EF21(wp.n, wp.d, wp.k, wp.gamma, wp.lam, total_rows=wp.N, device=device)
+            hm.load_shards(dev(wp.A), dev(wp.y), wp.row_offsets)
+            hm.init(B.INIT_COMPRESSED)
+            xm, gm, gim, _, _ = hm.get_state()
+            rows = torch.as_tensor(np.stack([inputs.minibatch_rows(9, t, wp.row_offsets, tau) for t in range(500)])).to(device)
+            hm.step_minibatches(rows[:20])
+            tm, lm = [], 0
+            for _ in range(5):
+                hm.set_state(xm, gm, gim)
+                flush_l2()
+                barrier()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                l0 = hm.launch_count
+                e0.record(); hm.step_minibatches(rows); e1.record()
+                barrier()
+                lm = hm.launch_count - l0
+                tm.append(slowest(e0.elapsed_time(e1)))
+            msm = statistics.median(tm)
+            others.append({"workload": f"stochastic EF21 (Algorithm 5) on configs[{HEADLINE}] {wp.name} Top-{wp.k}, tau = {tau}",
+                           "iterations_per_s": 500 / (msm * 1e-3), "us_per_iteration": msm / 500 * 1e3, "launches": lm,
+                           "device_status": hm.poll(), "f_end": hm.eval()[0]})
         line["workloads"] = others
         line["workloads_note"] = ("frac_of_hbm_peak = algorithmic bytes per iteration / time / measured copy peak (read + write); on the "
                                   "on-chip workloads it is not a DRAM figure (DRAM traffic per launch is the shards once), and a read-only "
