@@ -498,6 +498,30 @@ def test_two_handles_share_the_kernels(B, oracle32):
     assert ha.poll() == 0 and hb.poll() == 0
 
 
+@pytest.mark.parametrize("body", [1, 2], ids=["serving-warp", "whole-block"])
+@pytest.mark.parametrize("n,groups", [(5, 1), (20, 1), (32, 1), (20, 2), (24, 3)])
+def test_workers_naming_the_same_coordinate(n, groups, body, B, oracle32):
+    # `groups` distinct shards, each held by n / groups workers: in every iteration whole groups of workers send the same
+    # coordinate, so the per-coordinate sums in worker order have up to n terms (all 32 lanes of a polling round for
+    # n = 32; two or three interleaved groups of 8 to 10 otherwise)
+    m = 40
+    base = inputs.make_logistic("crowd", n=groups, d=96, N=groups * m, k=1, seed=7000 + n, features="gauss", flip=0.1, gamma=0.05, T=10)
+    w = inputs.make_logistic("crowd", n=n, d=96, N=n * m, k=1, seed=7000 + n, features="gauss", flip=0.1, gamma=0.05, T=10)
+    for i in range(n):
+        src = i % groups
+        w.A[i * m:(i + 1) * m] = base.A[src * m:(src + 1) * m]
+        w.y[i * m:(i + 1) * m] = base.y[src * m:(src + 1) * m]
+    h = make_gpu(w, k=1, path=2); h.set_persistent_body(body)
+    st = make_oracle_state(oracle32, w, k=1)
+    h.init(0); st.init(0)
+    sizes = []
+    for _ in range(12):
+        lockstep(h, st, oracle32, w, 1, k=1)
+        sizes.append(int(np.max(np.unique(st.idx[:, 0], return_counts=True)[1])))
+    assert min(sizes) >= n // groups, sizes
+    assert h.last_path == B.PATH_PERSISTENT and h.get_persistent_body() == body and h.poll() == 0
+
+
 def test_two_handles_on_two_streams_are_kept_apart(B):
     # 120 blocks each on 148 SMs: the two launches cannot be resident together, and each needs all of its clusters at
     # once.  The library orders a persistent launch after the device's previous one when the streams differ, so both
